@@ -1,0 +1,205 @@
+/*
+ * hadfl.h - C ABI of the HADFL round hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The method is HADFL (Cao et al., "HADFL: Heterogeneity-aware Decentralized Federated Learning
+ * Framework", arXiv 2111.08274).  N simulated heterogeneous devices each hold a flat parameter
+ * vector w (fp32, or bf16 storage) and an fp32 momentum vector m.  All replicas live in one
+ * device-memory arena: row i of w is device i's model, at w_ptr + i * row_stride_elems elements.
+ *
+ * One training round is the call sequence
+ *     hadfl_local_step   every device runs its own number E_i of local SGD steps
+ *                        (Eq. 3; Algorithm 1, "for e_k = 0 to E_k")
+ *     hadfl_select       N_p devices are drawn with the probability-based selection function
+ *                        (Eq. 8; Section "Heterogeneity-aware training strategy generation")
+ *     hadfl_aggregate    the selected replicas are averaged and the average is written back to
+ *                        them (Eq. 5; Algorithm 1, "partial synchronization")
+ *     hadfl_stats        per-replica squared norm and squared distance to a reference replica
+ *                        (diagnostics; not in the paper)
+ * and, when a model is wanted on the host (the coordinator's model backup, Section "Overall
+ * Design" item 9), hadfl_read_params.
+ *
+ * General rules
+ *   - Every function returns an int status: HADFL_OK, HADFL_ERR_INVALID (bad argument, duplicate or
+ *     out-of-range device id, k larger than the number of available devices, ...), HADFL_ERR_CUDA
+ *     (a CUDA call failed: hadfl_last_cuda_error gives the cudaError_t value), HADFL_ERR_STATE
+ *     (call not valid in the handle's state).  Nothing aborts and no kernel traps.  After
+ *     HADFL_ERR_INVALID the handle and the arena are unchanged.
+ *   - Pointer arguments are HOST pointers unless the comment says "device".  The caller owns every
+ *     buffer it passes; the library has copied what it needs when the call returns.
+ *   - All device work is enqueued on the one stream given at hadfl_init.  Calls return without
+ *     waiting for the GPU, except those marked "synchronises", which wait for that stream.
+ *   - A handle is not thread-safe.
+ *   - The synthetic gradient of parameter p of device i at its local step s is
+ *     grad_std * z, z a standard normal obtained by Box-Muller from the Philox4x32-10 block with
+ *     key = seed and counter = (p / 4, s mod 2^32, i, 'G' << 24 | s >> 32); lane p mod 4 of the
+ *     block.  It replaces forward/backward propagation, which is outside this library.
+ */
+#ifndef HADFL_H_
+#define HADFL_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HADFL_OK 0
+#define HADFL_ERR_INVALID 1
+#define HADFL_ERR_CUDA 2
+#define HADFL_ERR_STATE 3
+
+#define HADFL_MAX_DEVICES 32 /* largest N, and therefore largest k */
+
+#define HADFL_DTYPE_FP32 0 /* w stored as fp32 */
+#define HADFL_DTYPE_BF16 1 /* w stored as bf16, all arithmetic in fp32, one rounding per call */
+
+#define HADFL_WEIGHTS_UNIFORM 0 /* a_j = 1/k: Eq. 5 with K read as the number of selected devices */
+#define HADFL_WEIGHTS_VERSION 1 /* extension, not in the paper: a_j proportional to f(v_j) of Eq. 8 */
+
+typedef struct hadfl_handle hadfl_handle;
+
+typedef struct hadfl_config {
+  int32_t n_devices;        /* N, 1..HADFL_MAX_DEVICES */
+  int64_t n_params;         /* P >= 1, P <= 2^34 - 4 */
+  int32_t dtype;            /* HADFL_DTYPE_* */
+  float momentum;           /* mu of the local update */
+  float weight_decay;       /* wd of the local update */
+  float grad_std;           /* standard deviation of the synthetic gradients */
+  float init_std;           /* standard deviation of the initial model */
+  uint64_t seed;            /* key of the counter-based generator */
+  double version_scale;     /* versions are multiplied by this before Eq. 8 (1.0 = the paper) */
+  int32_t weight_mode;      /* HADFL_WEIGHTS_* */
+  void *w_ptr;              /* DEVICE pointer to the parameter arena, or NULL: the library
+                               allocates it (and the momentum arena) and frees it at destroy */
+  void *m_ptr;              /* DEVICE pointer to the fp32 momentum arena; NULL iff w_ptr is NULL */
+  int64_t row_stride_elems; /* elements between rows; 0 = P rounded up to a multiple of 32.
+                               Must be >= P and a multiple of 8.  Caller-owned arenas must be
+                               16-byte aligned, hold N * row_stride_elems elements each and outlive
+                               the handle. */
+  void *cuda_stream;        /* cudaStream_t on which all work is enqueued (NULL = default stream) */
+} hadfl_config;
+
+/* Algorithm 1, step 1 ("synchronize the initial models"): creates the handle on the current CUDA
+ * device, fills every row of w with the same w_(0)[p] = init_std * z(seed, p) and m with zeros
+ * (padding between rows too), and sets all versions and step counters to 0.  Asynchronous.
+ * On HADFL_ERR_CUDA *out is still a handle (so that the error code can be read) and must be
+ * destroyed; on other errors *out is NULL. */
+int hadfl_init(const hadfl_config *config, hadfl_handle **out);
+
+/* Waits for the stream, frees what the library allocated.  NULL is accepted. */
+int hadfl_destroy(hadfl_handle *h);
+
+/* Local update, Eq. 3 / Algorithm 1 (heterogeneity-aware local steps E_k): device device_ids[j]
+ * runs steps[j] >= 0 SGD steps on its own replica, in ONE kernel launch for all listed devices:
+ *     g = fma(wd, w, grad_std * z);  m = fma(mu, m, g);  w = fma(-lr, m, w)
+ * (momentum and weight decay follow the PyTorch SGD convention; Eq. 3 is mu = wd = 0).  w and m
+ * are read and written once per call whatever the step count.  Afterwards the version and the
+ * step counter of each listed device have grown by its step count.
+ * device_ids: n distinct ids in [0, N); 1 <= n <= N.  Asynchronous. */
+int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
+                     float lr);
+
+/* Probability-based selection, Eq. 8: P(i) = f(x_i) / sum_n f(x_n) over the available devices,
+ * x_i = versions[i] * version_scale, f the unit-variance Gaussian density about mu, mu the third
+ * quartile (linear interpolation) of the available x.  k distinct devices are drawn one after the
+ * other, each with probability proportional to f among those not yet drawn (uniformly if all
+ * remaining f underflow); out_selected receives them in draw order, which is also the ring order
+ * and the summation order of hadfl_aggregate.  The random stream is Philox4x32-10 keyed by `seed`
+ * with counter (t, 0, round, 'S' << 24): the result is a pure function of the arguments, the
+ * availability mask and version_scale.
+ * versions: N doubles, or NULL for the handle's own counters.  Host only; no GPU work. */
+int hadfl_select(hadfl_handle *h, int64_t round, const double *versions, uint64_t seed, int32_t k,
+                 int32_t *out_selected);
+
+/* Eq. 8 itself: out_P[i] = P(i) (0 for unavailable devices).  Host only. */
+int hadfl_select_probs(hadfl_handle *h, const double *versions, double *out_P);
+
+/* Partial aggregation, Eq. 5 / Algorithm 1 "partial synchronization", fused with the write-back:
+ *     acc = a_0 * w[selected[0]];  acc = fma(a_j, w[selected[j]], acc), j = 1..k-1;
+ *     w[selected[j]] = acc for all j          (one kernel, every element touched once)
+ * a_j = 1/k, or the version-dependent weights of weight_mode 1 computed from `versions` (N doubles,
+ * NULL = the handle's counters).  Momentum is not touched.  Afterwards every selected device carries
+ * the largest version among them.  selected: k distinct ids, 1 <= k <= N.  Asynchronous. */
+int hadfl_aggregate(hadfl_handle *h, const int32_t *selected, int32_t k, const double *versions);
+
+/* The weights a_j that hadfl_aggregate would use (out_a: k floats).  Host only. */
+int hadfl_aggregation_weights(hadfl_handle *h, const int32_t *selected, int32_t k,
+                              const double *versions, float *out_a);
+
+/* Global synchronisation, Algorithm 1 "send w to devices whose Flag = 0": the parameters of
+ * device src overwrite those of the n devices dst_ids (distinct, none equal to src, n may be 0),
+ * which also take its version.  One kernel: one read and n writes per element.  Asynchronous. */
+int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n);
+
+/* Per-replica statistics (not in the paper; diagnostics of how far the replicas have drifted):
+ * out_norm2[i] = sum_p w_i[p]^2, out_div2[i] = sum_p (w_i[p] - w_ref[p])^2, N floats each.
+ * Deterministic: fixed grid, fixed summation order, fp32 within a chunk, fp64 above.
+ * hadfl_stats = enqueue + read; hadfl_stats_read synchronises and returns the last enqueued result. */
+int hadfl_stats_enqueue(hadfl_handle *h, int32_t ref_device);
+int hadfl_stats_read(hadfl_handle *h, float *out_norm2, float *out_div2);
+int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *out_div2);
+
+/* Model backup (Section "Overall Design", item 9) and checkpointing.  `count` elements starting at
+ * parameter 0 of device_id; bf16 storage is widened to / rounded from fp32 (nearest even).
+ * Reads synchronise; writes are ordered on the stream and have consumed src on return. */
+int hadfl_read_params(hadfl_handle *h, int32_t device_id, float *dst, int64_t count);
+int hadfl_read_momentum(hadfl_handle *h, int32_t device_id, float *dst, int64_t count);
+int hadfl_write_params(hadfl_handle *h, int32_t device_id, const float *src, int64_t count);
+int hadfl_write_momentum(hadfl_handle *h, int32_t device_id, const float *src, int64_t count);
+
+/* Versions v_i ("actual parameter version of device i", Section "Runtime information prediction")
+ * and per-device step counters (the index into each device's gradient stream).  N entries each;
+ * either pointer may be NULL.  Restoring w, m, versions and step counters resumes a run exactly. */
+int hadfl_get_versions(hadfl_handle *h, uint32_t *versions, uint64_t *step_counts);
+int hadfl_set_versions(hadfl_handle *h, const uint32_t *versions, const uint64_t *step_counts);
+
+/* The set of available devices N_avl over which Eq. 8 normalises (liveness monitor, Section
+ * "Overall Design" item 1).  mask: N bytes, non-zero = available; NULL = all. */
+int hadfl_set_available(hadfl_handle *h, const uint8_t *mask);
+
+/* Waits for the handle's stream. */
+int hadfl_synchronize(hadfl_handle *h);
+
+/* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
+int hadfl_last_cuda_error(const hadfl_handle *h);
+
+/* Number of kernels this handle has launched so far. */
+uint64_t hadfl_launch_count(const hadfl_handle *h);
+
+/* Row stride, in elements, of the handle's arenas. */
+int64_t hadfl_row_stride(const hadfl_handle *h);
+
+/* ---- host-only functions (no handle, no GPU) ------------------------------------------------- */
+
+/* Eq. 8 on plain arrays: x (n doubles, already scaled), avail (n bytes or NULL), out_P (n). */
+int hadfl_selection_probs(const double *x, const uint8_t *avail, int32_t n, double *out_P);
+
+/* The draw of hadfl_select on plain arrays. */
+int hadfl_selection_draw(const double *x, const uint8_t *avail, int32_t n, int64_t round,
+                         uint64_t seed, int32_t k, int32_t *out_selected);
+
+/* Runtime version prediction, Eq. 7 (Brown's double exponential smoothing, 0 < alpha < 1):
+ * v1_j = alpha v_j + (1-alpha) v1_{j-1}, v2_j = alpha v1_j + (1-alpha) v2_{j-1}, both started at
+ * v_0; prediction m rounds after the last observation = (2 v1 - v2) + alpha/(1-alpha) (v1 - v2) m.
+ * series: n_obs >= 1 observed versions of one device.  Feeds the `versions` argument of
+ * hadfl_select when the coordinator plans with predicted instead of actual versions. */
+int hadfl_predict_version(const double *series, int32_t n_obs, double alpha, double m,
+                          double *out_prediction);
+
+/* ---- diagnostics of the on-device generator (used by the tests) -------------------------- */
+
+/* Philox4x32-10 on the GPU: counters (n x 4 words), key (2 words) -> out_words (n x 4).
+ * Host pointers; allocates temporaries; synchronises. */
+int hadfl_debug_philox(hadfl_handle *h, const uint32_t *counters, const uint32_t *key, int64_t n,
+                       uint32_t *out_words);
+
+/* The normals the local-update kernel draws for device `device` at step `step` for the n column
+ * groups `groups` (out_z: n x 4 floats), and (which = 1) those of the initial model.
+ * Host pointers; allocates temporaries; synchronises. */
+int hadfl_debug_normals(hadfl_handle *h, int32_t which, const uint32_t *groups, int64_t n,
+                        uint64_t step, uint32_t device, float *out_z);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HADFL_H_ */
