@@ -1,0 +1,519 @@
+// C ABI of the HADFL round hot path (see include/hadfl.h): handle, argument checks, version
+// bookkeeping, kernel launches.  Every step of the path runs in the kernels of kernels.cuh or in
+// the host planning arithmetic of selection.cpp; there is no other implementation to fall back to.
+#include "../../include/hadfl.h"
+
+#include <cuda_runtime.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+#include "selection.h"
+
+using namespace hadfl;
+
+struct hadfl_handle {
+  hadfl_config cfg;
+  int64_t stride = 0;
+  void *w = nullptr;
+  float *m = nullptr;
+  bool own_arena = false;
+  cudaStream_t stream = nullptr;
+  int device = 0;
+  int sm_count = 0;
+  PhiloxKeys keys;
+  uint32_t version[kMaxDevices];
+  uint64_t step_count[kMaxDevices];
+  uint8_t avail[kMaxDevices];
+  // K3 scratch
+  double *d_partials = nullptr;
+  unsigned int *d_ticket = nullptr;
+  float *d_stats = nullptr;
+  int stats_lanes = 0;  // blocks per row of the statistics kernel
+  bool stats_valid = false;
+  int last_cuda_error = 0;
+  uint64_t launches = 0;
+};
+
+namespace {
+
+constexpr int kStatsU = 4;  // column groups per thread and chunk in the statistics kernel
+
+#define HADFL_CUDA(h, expr)                       \
+  do {                                            \
+    cudaError_t e_ = (expr);                      \
+    if (e_ != cudaSuccess) {                      \
+      (h)->last_cuda_error = (int)e_;             \
+      return HADFL_ERR_CUDA;                      \
+    }                                             \
+  } while (0)
+
+// Makes the handle's device current for the duration of a call.
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+inline size_t elem_size(const hadfl_handle *h) { return h->cfg.dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
+
+inline int64_t n_groups(const hadfl_handle *h) { return (h->cfg.n_params + 3) / 4; }
+
+bool distinct_ids(const hadfl_handle *h, const int32_t *ids, int n) {
+  if (!ids || n < 1 || n > h->cfg.n_devices) return false;
+  uint32_t seen = 0;
+  for (int j = 0; j < n; ++j) {
+    if (ids[j] < 0 || ids[j] >= h->cfg.n_devices) return false;
+    if (seen & (1u << ids[j])) return false;
+    seen |= 1u << ids[j];
+  }
+  return true;
+}
+
+void scaled_versions(const hadfl_handle *h, const double *versions, double *x) {
+  for (int i = 0; i < h->cfg.n_devices; ++i)
+    x[i] = (versions ? versions[i] : (double)h->version[i]) * h->cfg.version_scale;
+}
+
+int check_launch(hadfl_handle *h) {
+  HADFL_CUDA(h, cudaGetLastError());
+  ++h->launches;
+  return HADFL_OK;
+}
+
+template <typename WT>
+int launch_init(hadfl_handle *h) {
+  const int64_t groups = h->stride / 4;
+  const unsigned blocks = (unsigned)((groups + kThreads - 1) / kThreads);
+  k_init<WT><<<blocks, kThreads, 0, h->stream>>>((WT *)h->w, h->m, h->stride, h->cfg.n_params,
+                                                 h->cfg.n_devices, h->keys, h->cfg.init_std);
+  return check_launch(h);
+}
+
+template <typename WT>
+int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
+  const unsigned blocks = (unsigned)((n_groups(h) + kThreads - 1) / kThreads);
+  k_local_step<WT, NormalsFast><<<blocks, kThreads, 0, h->stream>>>(
+      (WT *)h->w, h->m, h->stride, h->cfg.n_params, a, h->keys, lr, h->cfg.momentum,
+      h->cfg.weight_decay, h->cfg.grad_std);
+  return check_launch(h);
+}
+
+template <typename WT, int KR, int U>
+int launch_combine_as(hadfl_handle *h, const CombineArgs &c) {
+  const int64_t per_block = (int64_t)kThreads * U;
+  const unsigned blocks = (unsigned)((n_groups(h) + per_block - 1) / per_block);
+  k_combine<WT, KR, U><<<blocks, kThreads, 0, h->stream>>>((WT *)h->w, h->stride,
+                                                            h->cfg.n_params, c);
+  return check_launch(h);
+}
+
+template <typename WT>
+int launch_combine(hadfl_handle *h, const CombineArgs &c) {
+  switch (c.nr) {
+    case 1: return launch_combine_as<WT, 1, 4>(h, c);
+    case 2: return launch_combine_as<WT, 2, 4>(h, c);
+    case 3: return launch_combine_as<WT, 3, 2>(h, c);
+    case 4: return launch_combine_as<WT, 4, 2>(h, c);
+    case 8: return launch_combine_as<WT, 8, 1>(h, c);
+    case 16: return launch_combine_as<WT, 16, 1>(h, c);
+    default: return launch_combine_as<WT, 0, 1>(h, c);
+  }
+}
+
+template <typename WT>
+int launch_stats(hadfl_handle *h, int ref) {
+  k_stats<WT, kStatsU><<<h->stats_lanes * h->cfg.n_devices, kThreads, 0, h->stream>>>(
+      (const WT *)h->w, h->stride, h->cfg.n_params, h->cfg.n_devices, ref, h->stats_lanes,
+      h->d_partials, h->d_ticket, h->d_stats);
+  return check_launch(h);
+}
+
+int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool momentum) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (!dst || id < 0 || id >= h->cfg.n_devices || count < 0 || count > h->cfg.n_params)
+    return HADFL_ERR_INVALID;
+  DeviceGuard guard(h->device);
+  if (count == 0) {
+    HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+    return HADFL_OK;
+  }
+  if (momentum || h->cfg.dtype == HADFL_DTYPE_FP32) {
+    const float *src = (momentum ? h->m : (const float *)h->w) + (int64_t)id * h->stride;
+    HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost,
+                                  h->stream));
+    HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+    return HADFL_OK;
+  }
+  std::vector<uint16_t> tmp((size_t)count);
+  const uint16_t *src = (const uint16_t *)h->w + (int64_t)id * h->stride;
+  HADFL_CUDA(h, cudaMemcpyAsync(tmp.data(), src, 2 * (size_t)count, cudaMemcpyDeviceToHost, h->stream));
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  for (int64_t p = 0; p < count; ++p) {
+    const uint32_t bits = (uint32_t)tmp[(size_t)p] << 16;
+    memcpy(dst + p, &bits, 4);
+  }
+  return HADFL_OK;
+}
+
+uint16_t bf16_bits_rn(float v) {
+  uint32_t bits;
+  memcpy(&bits, &v, 4);
+  if ((bits & 0x7F800000u) == 0x7F800000u) return (uint16_t)((bits >> 16) | ((bits & 0x007FFFFFu) ? 0x40u : 0u));
+  return (uint16_t)((bits + 0x7FFFu + ((bits >> 16) & 1u)) >> 16);
+}
+
+int write_row(hadfl_handle *h, int32_t id, const float *src, int64_t count, bool momentum) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (!src || id < 0 || id >= h->cfg.n_devices || count < 0 || count > h->cfg.n_params)
+    return HADFL_ERR_INVALID;
+  if (count == 0) return HADFL_OK;
+  DeviceGuard guard(h->device);
+  // The copy is ordered on the stream; waiting for it lets the caller reuse src at once.
+  if (momentum || h->cfg.dtype == HADFL_DTYPE_FP32) {
+    float *dst = (momentum ? h->m : (float *)h->w) + (int64_t)id * h->stride;
+    HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyHostToDevice,
+                                  h->stream));
+    HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+    return HADFL_OK;
+  }
+  std::vector<uint16_t> tmp((size_t)count);
+  for (int64_t p = 0; p < count; ++p) tmp[(size_t)p] = bf16_bits_rn(src[p]);
+  uint16_t *dst = (uint16_t *)h->w + (int64_t)id * h->stride;
+  HADFL_CUDA(h, cudaMemcpyAsync(dst, tmp.data(), 2 * (size_t)count, cudaMemcpyHostToDevice, h->stream));
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  return HADFL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
+  if (!cfg || !out) return HADFL_ERR_INVALID;
+  *out = nullptr;
+  if (cfg->n_devices < 1 || cfg->n_devices > HADFL_MAX_DEVICES) return HADFL_ERR_INVALID;
+  if (cfg->n_params < 1 || cfg->n_params > ((int64_t)1 << 34) - 4) return HADFL_ERR_INVALID;
+  if (cfg->dtype != HADFL_DTYPE_FP32 && cfg->dtype != HADFL_DTYPE_BF16) return HADFL_ERR_INVALID;
+  if (cfg->weight_mode != HADFL_WEIGHTS_UNIFORM && cfg->weight_mode != HADFL_WEIGHTS_VERSION)
+    return HADFL_ERR_INVALID;
+  if ((cfg->w_ptr == nullptr) != (cfg->m_ptr == nullptr)) return HADFL_ERR_INVALID;
+  if (!(cfg->version_scale > 0.0)) return HADFL_ERR_INVALID;
+  int64_t stride = cfg->row_stride_elems;
+  if (stride == 0) stride = (cfg->n_params + 31) / 32 * 32;
+  if (stride < cfg->n_params || stride % 8 != 0) return HADFL_ERR_INVALID;
+  if (cfg->w_ptr && (((uintptr_t)cfg->w_ptr | (uintptr_t)cfg->m_ptr) & 15u)) return HADFL_ERR_INVALID;
+
+  hadfl_handle *h = new (std::nothrow) hadfl_handle;
+  if (!h) return HADFL_ERR_STATE;
+  h->cfg = *cfg;
+  h->stride = stride;
+  h->stream = (cudaStream_t)cfg->cuda_stream;
+  h->keys = expand_keys(cfg->seed);
+  for (int i = 0; i < kMaxDevices; ++i) {
+    h->version[i] = 0;
+    h->step_count[i] = 0;
+    h->avail[i] = 1;
+  }
+  // From here on failures are CUDA failures; the handle is returned so that the caller can read
+  // the error code, and must still be destroyed.
+  *out = h;
+  HADFL_CUDA(h, cudaGetDevice(&h->device));
+  HADFL_CUDA(h, cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device));
+  const size_t elems = (size_t)cfg->n_devices * (size_t)stride;
+  if (!cfg->w_ptr) {
+    h->own_arena = true;
+    HADFL_CUDA(h, cudaMalloc(&h->w, elems * elem_size(h)));
+    HADFL_CUDA(h, cudaMalloc((void **)&h->m, elems * sizeof(float)));
+  } else {
+    h->w = cfg->w_ptr;
+    h->m = (float *)cfg->m_ptr;
+  }
+  // Statistics grid: one wave of resident blocks (8 blocks of 256 threads per SM), split evenly
+  // over the rows; never more blocks per row than there are column chunks.
+  const int64_t chunks = (n_groups(h) + kThreads * kStatsU - 1) / (kThreads * kStatsU);
+  int64_t lanes = ((int64_t)h->sm_count * 8 + cfg->n_devices - 1) / cfg->n_devices;
+  if (lanes > chunks) lanes = chunks;
+  h->stats_lanes = (int)lanes;
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_partials,
+                           sizeof(double) * 2 * (size_t)cfg->n_devices * (size_t)lanes));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_ticket, sizeof(unsigned int)));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
+  return cfg->dtype == HADFL_DTYPE_BF16 ? launch_init<__nv_bfloat16>(h) : launch_init<float>(h);
+}
+
+int hadfl_destroy(hadfl_handle *h) {
+  if (!h) return HADFL_OK;
+  DeviceGuard guard(h->device);
+  cudaStreamSynchronize(h->stream);
+  if (h->own_arena) {
+    cudaFree(h->w);
+    cudaFree(h->m);
+  }
+  cudaFree(h->d_partials);
+  cudaFree(h->d_ticket);
+  cudaFree(h->d_stats);
+  delete h;
+  return HADFL_OK;
+}
+
+int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
+                     float lr) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (!steps || !distinct_ids(h, device_ids, n)) return HADFL_ERR_INVALID;
+  for (int j = 0; j < n; ++j)
+    if (steps[j] < 0) return HADFL_ERR_INVALID;
+  LocalStepArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = n;
+  for (int j = 0; j < n; ++j) {
+    const uint64_t base = h->step_count[device_ids[j]];
+    if ((base + (uint64_t)steps[j]) >> 56) return HADFL_ERR_STATE;  // the counter's stream has 2^56 steps
+    a.row[j] = device_ids[j];
+    a.steps[j] = steps[j];
+    a.base_lo[j] = (uint32_t)base;
+    a.base_hi[j] = (uint32_t)(base >> 32);
+  }
+  DeviceGuard guard(h->device);
+  const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_local_step<__nv_bfloat16>(h, a, lr)
+                                                  : launch_local_step<float>(h, a, lr);
+  if (rc != HADFL_OK) return rc;
+  for (int j = 0; j < n; ++j) {
+    h->step_count[device_ids[j]] += (uint64_t)steps[j];
+    h->version[device_ids[j]] += (uint32_t)steps[j];
+  }
+  return HADFL_OK;
+}
+
+int hadfl_select(hadfl_handle *h, int64_t round, const double *versions, uint64_t seed, int32_t k,
+                 int32_t *out_selected) {
+  if (!h || !out_selected) return HADFL_ERR_INVALID;
+  double x[kMaxDevices];
+  scaled_versions(h, versions, x);
+  return selection_draw(x, h->avail, h->cfg.n_devices, round, seed, k, out_selected)
+             ? HADFL_OK
+             : HADFL_ERR_INVALID;
+}
+
+int hadfl_select_probs(hadfl_handle *h, const double *versions, double *out_P) {
+  if (!h || !out_P) return HADFL_ERR_INVALID;
+  double x[kMaxDevices];
+  scaled_versions(h, versions, x);
+  return selection_probs(x, h->avail, h->cfg.n_devices, out_P) ? HADFL_OK : HADFL_ERR_INVALID;
+}
+
+int hadfl_aggregation_weights(hadfl_handle *h, const int32_t *selected, int32_t k,
+                              const double *versions, float *out_a) {
+  if (!h || !out_a || !distinct_ids(h, selected, k)) return HADFL_ERR_INVALID;
+  double x[kMaxDevices];
+  scaled_versions(h, versions, x);
+  aggregation_weights(h->cfg.weight_mode, x, h->avail, h->cfg.n_devices, selected, k, out_a);
+  return HADFL_OK;
+}
+
+int hadfl_aggregate(hadfl_handle *h, const int32_t *selected, int32_t k, const double *versions) {
+  if (!h || !distinct_ids(h, selected, k)) return HADFL_ERR_INVALID;
+  CombineArgs c;
+  memset(&c, 0, sizeof(c));
+  c.nr = c.nw = k;
+  double x[kMaxDevices];
+  scaled_versions(h, versions, x);
+  aggregation_weights(h->cfg.weight_mode, x, h->avail, h->cfg.n_devices, selected, k, c.a);
+  for (int j = 0; j < k; ++j) c.rd[j] = c.wr[j] = selected[j];
+  if (k > 1) {  // a single selected device is a no-op (a_0 = 1): nothing to launch
+    DeviceGuard guard(h->device);
+    const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_combine<__nv_bfloat16>(h, c)
+                                                    : launch_combine<float>(h, c);
+    if (rc != HADFL_OK) return rc;
+  }
+  uint32_t vmax = 0;
+  for (int j = 0; j < k; ++j) vmax = h->version[selected[j]] > vmax ? h->version[selected[j]] : vmax;
+  for (int j = 0; j < k; ++j) h->version[selected[j]] = vmax;
+  return HADFL_OK;
+}
+
+int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n) {
+  if (!h || src < 0 || src >= h->cfg.n_devices || n < 0) return HADFL_ERR_INVALID;
+  if (n == 0) return HADFL_OK;
+  if (!distinct_ids(h, dst_ids, n)) return HADFL_ERR_INVALID;
+  for (int j = 0; j < n; ++j)
+    if (dst_ids[j] == src) return HADFL_ERR_INVALID;
+  CombineArgs c;
+  memset(&c, 0, sizeof(c));
+  c.nr = 1;
+  c.nw = n;
+  c.rd[0] = src;
+  c.a[0] = 1.0f;
+  for (int j = 0; j < n; ++j) c.wr[j] = dst_ids[j];
+  DeviceGuard guard(h->device);
+  const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_combine<__nv_bfloat16>(h, c)
+                                                  : launch_combine<float>(h, c);
+  if (rc != HADFL_OK) return rc;
+  for (int j = 0; j < n; ++j) h->version[dst_ids[j]] = h->version[src];
+  return HADFL_OK;
+}
+
+int hadfl_stats_enqueue(hadfl_handle *h, int32_t ref_device) {
+  if (!h || ref_device < 0 || ref_device >= h->cfg.n_devices) return HADFL_ERR_INVALID;
+  DeviceGuard guard(h->device);
+  const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_stats<__nv_bfloat16>(h, ref_device)
+                                                  : launch_stats<float>(h, ref_device);
+  if (rc == HADFL_OK) h->stats_valid = true;
+  return rc;
+}
+
+int hadfl_stats_read(hadfl_handle *h, float *out_norm2, float *out_div2) {
+  if (!h || !out_norm2 || !out_div2) return HADFL_ERR_INVALID;
+  if (!h->stats_valid) return HADFL_ERR_STATE;
+  DeviceGuard guard(h->device);
+  float buf[2 * kMaxDevices];
+  const int n = h->cfg.n_devices;
+  HADFL_CUDA(h, cudaMemcpyAsync(buf, h->d_stats, sizeof(float) * 2 * (size_t)n,
+                                cudaMemcpyDeviceToHost, h->stream));
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  memcpy(out_norm2, buf, sizeof(float) * (size_t)n);
+  memcpy(out_div2, buf + n, sizeof(float) * (size_t)n);
+  return HADFL_OK;
+}
+
+int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *out_div2) {
+  if (!h || !out_norm2 || !out_div2) return HADFL_ERR_INVALID;
+  const int rc = hadfl_stats_enqueue(h, ref_device);
+  return rc != HADFL_OK ? rc : hadfl_stats_read(h, out_norm2, out_div2);
+}
+
+int hadfl_read_params(hadfl_handle *h, int32_t id, float *dst, int64_t count) {
+  return read_row(h, id, dst, count, false);
+}
+int hadfl_read_momentum(hadfl_handle *h, int32_t id, float *dst, int64_t count) {
+  return read_row(h, id, dst, count, true);
+}
+int hadfl_write_params(hadfl_handle *h, int32_t id, const float *src, int64_t count) {
+  return write_row(h, id, src, count, false);
+}
+int hadfl_write_momentum(hadfl_handle *h, int32_t id, const float *src, int64_t count) {
+  return write_row(h, id, src, count, true);
+}
+
+int hadfl_get_versions(hadfl_handle *h, uint32_t *versions, uint64_t *step_counts) {
+  if (!h) return HADFL_ERR_INVALID;
+  for (int i = 0; i < h->cfg.n_devices; ++i) {
+    if (versions) versions[i] = h->version[i];
+    if (step_counts) step_counts[i] = h->step_count[i];
+  }
+  return HADFL_OK;
+}
+
+int hadfl_set_versions(hadfl_handle *h, const uint32_t *versions, const uint64_t *step_counts) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (step_counts)
+    for (int i = 0; i < h->cfg.n_devices; ++i)
+      if (step_counts[i] >> 56) return HADFL_ERR_INVALID;
+  for (int i = 0; i < h->cfg.n_devices; ++i) {
+    if (versions) h->version[i] = versions[i];
+    if (step_counts) h->step_count[i] = step_counts[i];
+  }
+  return HADFL_OK;
+}
+
+int hadfl_set_available(hadfl_handle *h, const uint8_t *mask) {
+  if (!h) return HADFL_ERR_INVALID;
+  for (int i = 0; i < h->cfg.n_devices; ++i) h->avail[i] = mask ? (mask[i] ? 1 : 0) : 1;
+  return HADFL_OK;
+}
+
+int hadfl_synchronize(hadfl_handle *h) {
+  if (!h) return HADFL_ERR_INVALID;
+  DeviceGuard guard(h->device);
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  return HADFL_OK;
+}
+
+int hadfl_last_cuda_error(const hadfl_handle *h) { return h ? h->last_cuda_error : 0; }
+uint64_t hadfl_launch_count(const hadfl_handle *h) { return h ? h->launches : 0; }
+int64_t hadfl_row_stride(const hadfl_handle *h) { return h ? h->stride : 0; }
+
+int hadfl_selection_probs(const double *x, const uint8_t *avail, int32_t n, double *out_P) {
+  if (!x || !out_P || n < 1 || n > HADFL_MAX_DEVICES) return HADFL_ERR_INVALID;
+  return selection_probs(x, avail, n, out_P) ? HADFL_OK : HADFL_ERR_INVALID;
+}
+
+int hadfl_selection_draw(const double *x, const uint8_t *avail, int32_t n, int64_t round,
+                         uint64_t seed, int32_t k, int32_t *out_selected) {
+  if (!x || !out_selected || n < 1 || n > HADFL_MAX_DEVICES) return HADFL_ERR_INVALID;
+  return selection_draw(x, avail, n, round, seed, k, out_selected) ? HADFL_OK : HADFL_ERR_INVALID;
+}
+
+int hadfl_predict_version(const double *series, int32_t n_obs, double alpha, double m,
+                          double *out_prediction) {
+  if (!series || !out_prediction || n_obs < 1 || !(alpha > 0.0 && alpha < 1.0)) return HADFL_ERR_INVALID;
+  *out_prediction = predict_version(series, n_obs, alpha, m);
+  return HADFL_OK;
+}
+
+int hadfl_debug_philox(hadfl_handle *h, const uint32_t *counters, const uint32_t *key, int64_t n,
+                       uint32_t *out_words) {
+  if (!h || !counters || !key || !out_words || n < 0) return HADFL_ERR_INVALID;
+  if (n == 0) return HADFL_OK;
+  DeviceGuard guard(h->device);
+  uint32_t *d_in = nullptr, *d_out = nullptr;
+  const size_t bytes = sizeof(uint32_t) * 4 * (size_t)n;
+  HADFL_CUDA(h, cudaMalloc((void **)&d_in, bytes));
+  cudaError_t e = cudaMalloc((void **)&d_out, bytes);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_in, counters, bytes, cudaMemcpyHostToDevice, h->stream);
+  if (e == cudaSuccess) {
+    const PhiloxKeys keys = expand_keys(((uint64_t)key[1] << 32) | key[0]);
+    k_debug_philox<<<(unsigned)((n + 255) / 256), 256, 0, h->stream>>>(d_in, keys, n, d_out);
+    e = cudaGetLastError();
+    ++h->launches;
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(out_words, d_out, bytes, cudaMemcpyDeviceToHost, h->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  cudaFree(d_in);
+  cudaFree(d_out);
+  HADFL_CUDA(h, e);
+  return HADFL_OK;
+}
+
+int hadfl_debug_normals(hadfl_handle *h, int32_t which, const uint32_t *groups, int64_t n,
+                        uint64_t step, uint32_t device, float *out_z) {
+  if (!h || !groups || !out_z || n < 0 || (which != 0 && which != 1)) return HADFL_ERR_INVALID;
+  if (n == 0) return HADFL_OK;
+  DeviceGuard guard(h->device);
+  uint32_t *d_in = nullptr;
+  float4 *d_out = nullptr;
+  HADFL_CUDA(h, cudaMalloc((void **)&d_in, sizeof(uint32_t) * (size_t)n));
+  cudaError_t e = cudaMalloc((void **)&d_out, sizeof(float4) * (size_t)n);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(d_in, groups, sizeof(uint32_t) * (size_t)n, cudaMemcpyHostToDevice, h->stream);
+  if (e == cudaSuccess) {
+    const unsigned blocks = (unsigned)((n + 255) / 256);
+    if (which == 0)
+      k_debug_normals<NormalsFast><<<blocks, 256, 0, h->stream>>>(
+          d_in, n, (uint32_t)step, device, kTagGrad | ((uint32_t)(step >> 32) & 0xFFFFFFu), h->keys, d_out);
+    else
+      k_debug_normals<NormalsAccurate><<<blocks, 256, 0, h->stream>>>(d_in, n, 0u, 0u, kTagInit,
+                                                                       h->keys, d_out);
+    e = cudaGetLastError();
+    ++h->launches;
+  }
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(out_z, d_out, sizeof(float4) * (size_t)n, cudaMemcpyDeviceToHost, h->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  cudaFree(d_in);
+  cudaFree(d_out);
+  HADFL_CUDA(h, e);
+  return HADFL_OK;
+}
+
+}  // extern "C"
