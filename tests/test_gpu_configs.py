@@ -1,0 +1,128 @@
+"""End-to-end parity of the five workloads: the CUDA path against the CPU oracle, round by round.
+
+Selections and version / step counters must agree exactly in every round.  Parameters are compared
+within max|gpu - cpu| <= 2e-6 * max|x|: on the whole arena where the oracle finishes in seconds,
+otherwise (the full-size vectors) on a column sample - the first and last groups of every row plus
+random groups in between - which the oracle can follow on its own because every operation of the
+round is elementwise in the column index.  bf16 storage: almost all elements equal, the others
+within two bf16 steps (a last-bit difference of a gradient normal can move a rounding decision)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_common import TOL_REL, assert_close_params, bf16_ulp, require_gpu
+from oracle_driver import make_sim, oracle_round
+from paper_2111_08274_b200 import runtime, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def columns_of(groups, n_params):
+    cols = (4 * groups.astype(np.int64)[:, None] + np.arange(4)[None, :]).reshape(-1)
+    return cols, cols < n_params
+
+
+def compare_sample(arena, sim, groups, what):
+    wl = arena.wl
+    cols, live = columns_of(groups, wl.n_params)
+    idx = torch.from_numpy(np.where(live, cols, 0)).to(arena.device)
+    worst = 0.0
+    for i in range(wl.n_devices):
+        got = arena.w[i, idx].float().cpu().numpy()[live]
+        want = sim.read_cols(i)[live]
+        if wl.dtype == 0:
+            worst = max(worst, assert_close_params(got, want, "%s w[%d]" % (what, i)))
+        else:
+            # A rounding decision that went the other way leaves a difference of one bf16 step of the
+            # value at that time, which persists while the value itself moves on: bound it by two
+            # steps at the largest magnitude in the row, and require such elements to be rare.
+            assert np.abs(got - want).max() <= 2 * bf16_ulp(np.abs(want).max()), (what, i)
+            assert np.mean(got != want) < 0.01, (what, i)
+        gm = arena.m[i, idx].cpu().numpy()[live]
+        # momentum sees the generator's error directly (not scaled by lr); with bf16 storage a
+        # moved rounding of w also enters through weight decay
+        m_tol = wl.grad_std * 1e-5 / (1.0 - wl.momentum) + (wl.weight_decay * 0.004 / (1.0 - wl.momentum) if wl.dtype else 0.0)
+        assert np.abs(gm - sim.read_momentum_cols(i)[live]).max() <= m_tol, (what, i)
+    return worst
+
+
+def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=()):
+    arena = runtime.Arena(wl)
+    sim = make_sim(oracle, wl, groups)
+    full = groups is None
+    g = np.arange((wl.n_params + 3) // 4, dtype=np.uint32) if full else groups
+    worst = 0.0
+    for r in range(wl.rounds):
+        sel = arena.run_round(r)
+        want_sel = oracle_round(sim, wl, r)
+        assert np.array_equal(sel, want_sel), "round %d: selection %s != %s" % (r, sel, want_sel)
+        v, s = arena.h.get_versions()
+        ov, os_ = sim.get_versions()
+        assert np.array_equal(v, ov) and np.array_equal(s, os_), "round %d: counters differ" % r
+        if r in check_rounds or r == wl.rounds - 1:
+            worst = max(worst, compare_sample(arena, sim, g, "%s round %d" % (wl.name, r)))
+        if full and (r in stats_rounds or r == wl.rounds - 1):
+            n2, d2 = arena.h.stats_read()
+            wn2, wd2 = sim.stats(int(sel[0]))
+            assert np.allclose(n2, wn2, rtol=1e-5) and np.allclose(d2, wd2, rtol=1e-5, atol=1e-12)
+    n2, d2 = arena.h.stats_read()
+    assert np.all(np.isfinite(n2)) and np.all(d2 >= 0) and d2[int(sel[0])] == 0.0
+    launches = arena.h.launch_count()
+    arena.close()
+    print("%s: %d rounds ok, max err / max|x| = %.2e, %d launches" % (wl.name, wl.rounds, worst, launches))
+    return worst
+
+
+def test_c1_full_arena_every_round(oracle):
+    wl = workloads.c1()
+    run_and_compare(oracle, wl, None, check_rounds=range(wl.rounds), stats_rounds=range(wl.rounds))
+
+
+def test_c1_ragged_tail_full_arena(oracle):
+    """The same workload on a vector whose length is not a multiple of 4 and spans several blocks."""
+    wl = workloads.shrink(workloads.c1(), 100_003)
+    run_and_compare(oracle, wl, None, check_rounds=(0, 4))
+
+
+def test_c2_full_size_sampled_columns(oracle):
+    wl = workloads.c2()
+    groups = workloads.sample_groups(wl.n_params, 30_000, 1024, seed=2)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24))
+
+
+def test_c2_shrunk_full_arena(oracle):
+    wl = workloads.shrink(workloads.c2(), 50_002, rounds=8)
+    run_and_compare(oracle, wl, None, check_rounds=range(8), stats_rounds=range(8))
+
+
+def test_c3_full_size_sampled_columns(oracle):
+    wl = workloads.c3()
+    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=3)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 10, 49))
+
+
+@pytest.mark.parametrize("k", [2, 8, 16])
+def test_c4_full_size_sampled_columns(oracle, k):
+    wl = workloads.c4(k)
+    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=4 + k)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9))
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("log2_p", range(16, 28))
+def test_c5_bandwidth_sweep_sizes(oracle, log2_p, dtype):
+    for hetero in (False, True):
+        wl = workloads.c5(log2_p, dtype=dtype, hetero=hetero)
+        groups = workloads.sample_groups(wl.n_params, 256, 128, seed=log2_p)
+        run_and_compare(oracle, wl, groups, check_rounds=(0, 4, 99))
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_c5_smallest_size_full_arena_first_rounds(oracle, dtype):
+    wl = workloads.shrink(workloads.c5(16, dtype=dtype, hetero=True), 1 << 16, rounds=5)
+    run_and_compare(oracle, wl, None, check_rounds=range(5), stats_rounds=range(5))
