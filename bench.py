@@ -1,0 +1,338 @@
+"""Benchmark of the HADFL round hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+
+A "step" is one round of the whole hot path over one synthetic workload: local update of every
+device with its own step count (K1), selection (host), aggregation with write-back (K2), version
+update and per-replica statistics (K3).  Prints ONE JSON line (rank 0).
+
+  value     rounds/s with everything resident in HBM; timed with CUDA events on the library's
+            stream, barrier + synchronize on both sides, max over ranks.
+  e2e       the same rounds through the C ABI with HOST buffers: every round also reads the
+            statistics (2N floats) and the aggregated model (P floats, the coordinator's model
+            backup) into pinned host memory.
+  roofline  for the kernel with the largest share of the timed region: algorithmic bytes per
+            launch / average launch time (CUDA events around each launch), against the measured
+            copy bandwidth of this machine's B200s.
+  cpu_baseline  the CPU checker (single thread, as it stands) on a column sample of the same
+            workload, scaled to the full vector.
+
+N > 1 runs N independent replicas of the workload, one process per GPU (launched by torchrun):
+the path does not shard across GPUs and has no exchange step, so there is no collective in it.
+--impl reference times the CPU checker instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2111_08274_b200 import workloads  # noqa: E402
+
+METRIC = "aggregation_rounds_per_sec"
+UNIT = "rounds/s"
+FALLBACK_HBM_GBS = 6650.0
+ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to size its sample
+
+# DRAM bytes per (device, parameter) moved by one launch, from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same kernel;
+# traffic grows in proportion to the elements processed).  None = not captured for the kernel
+# as it stands.
+NCU_DRAM_BYTES_PER_ELEM = {"local_step": None, "aggregate": None, "stats": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def describe(wl):
+    steps = "uniform[%d,%d] per device per round" % (wl.steps_lo, wl.steps_hi) \
+        if wl.steps_rule == "uniform" else "fixed %s" % (list(wl.steps_fixed),)
+    return {"workload": wl.name, "n_devices": wl.n_devices, "n_params": wl.n_params, "k": wl.k,
+            "local_steps": steps, "lr": wl.lr, "momentum": wl.momentum,
+            "weight_decay": wl.weight_decay, "grad_std": wl.grad_std,
+            "storage": "bf16" if wl.dtype else "fp32",
+            "arena_bytes": wl.n_devices * wl.n_params * (6 if wl.dtype else 8),
+            "l2": "arena is larger than L2 (126 MB): no flush between rounds",
+            "multi_gpu": "replicas only (no sharding, no collective)"}
+
+
+def mean_steps_per_device(wl, rounds=8):
+    return float(np.mean([wl.steps_for_round(r).sum() for r in range(rounds)])) / wl.n_devices
+
+
+# ---- CPU checker timing ------------------------------------------------------------------------
+def time_oracle(wl, frac_cols, rounds):
+    """Rounds of the CPU checker on the first `frac_cols` of the column groups; returns
+    (seconds per full-vector round for each round, description of the sample)."""
+    import oracle
+    n_groups = (wl.n_params + 3) // 4
+    take = min(n_groups, max(64, int(n_groups * frac_cols)))
+    groups = np.arange(take, dtype=np.uint32)
+    sim = oracle.Sim(wl.n_devices, wl.n_params, dtype=wl.dtype, momentum=wl.momentum,
+                     weight_decay=wl.weight_decay, grad_std=wl.grad_std, init_std=wl.init_std,
+                     seed=wl.seed, version_scale=wl.version_scale, weight_mode=wl.weight_mode,
+                     groups=groups)
+    ids = wl.device_ids()
+    per_round = []
+    for r in range(rounds):
+        t0 = time.perf_counter()
+        sim.local_step(ids, wl.steps_for_round(r), wl.lr)
+        sel = sim.select(r, wl.k, wl.select_seed())
+        sim.aggregate(sel)
+        sim.stats(int(sel[0]))
+        per_round.append(time.perf_counter() - t0)
+    sim.close()
+    scale = n_groups / float(take)
+    what = "%d round(s) on the first %d of %d column groups (%.3f%% of the vector), scaled by %.1f" % (
+        rounds, take, n_groups, 100.0 / scale, scale)
+    return [t * scale for t in per_round], what
+
+
+def run_reference(args, wl):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    # Bounded sample: size the column sample so that the whole run takes about a minute.
+    total = args.warmup + args.steps
+    full_round_s = wl.n_devices * wl.n_params * mean_steps_per_device(wl) * ORACLE_NS_PER_ELEM_STEP
+    frac = min(1.0 / 8.0, 60.0 / (total * full_round_s))
+    times, what = time_oracle(wl, frac, total)
+    sec = float(np.mean(times[args.warmup:]))
+    value = 1.0 / sec
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": describe(wl),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---- clocks --------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs (NVML, read
+    only)."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+                bits = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def max_over_ranks(value, world):
+    """Max of a host scalar over all ranks (the job is as slow as its slowest rank)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ---- our arm ---------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2111_08274_b200 import runtime
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world:
+        raise SystemExit("--gpus %d does not match WORLD_SIZE %d (launch with torch.distributed.run)"
+                         % (args.gpus, world))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    runtime.ensure_built()
+
+    arena = runtime.Arena(wl, device="cuda:%d" % local)
+    h = arena.h
+    N, P, k = wl.n_devices, wl.n_params, wl.k
+    elem_w = 2 if wl.dtype else 4
+    warmup = max(args.warmup, 3)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    r = 0
+    for _ in range(warmup):
+        arena.run_round(r)
+        r += 1
+
+    K = args.steps
+    names = ("local_step", "aggregate", "stats")
+    ev = {n: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(K)] for n in names}
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(physical_gpu_index(local))
+    ids, seed = arena.ids, arena.select_seed
+    step_lists = [wl.steps_for_round(r + i) for i in range(K)]
+    barrier()
+    launches0 = h.launch_count()
+    sampler.start()
+    start.record()
+    for i in range(K):
+        a, b = ev["local_step"][i]
+        a.record(); h.local_step(ids, step_lists[i], wl.lr); b.record()
+        sel = h.select(r + i, k, seed)
+        a, b = ev["aggregate"][i]
+        a.record(); h.aggregate(sel); b.record()
+        a, b = ev["stats"][i]
+        a.record(); h.stats_enqueue(int(sel[0])); b.record()
+    end.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = h.launch_count() - launches0
+    r += K
+    elapsed_ms = max_over_ranks(start.elapsed_time(end), world)
+
+    kern_ms = {n: float(np.mean([a.elapsed_time(b) for a, b in ev[n]])) for n in names}
+    mean_steps = float(np.mean([s.sum() for s in step_lists])) / N
+    alg_bytes = {"local_step": N * P * (2 * elem_w + 8),       # read + write w and m, once per call
+                 "aggregate": 2 * k * P * elem_w,              # k rows read, k rows written
+                 "stats": N * P * elem_w}                      # every row read once
+    units = {"local_step": N * P, "aggregate": k * P, "stats": N * P}
+    peak, peak_kind = measured_peak()
+    kernels = {}
+    for n in names:
+        gbs = alg_bytes[n] / (kern_ms[n] * 1e-3) / 1e9
+        per_elem = NCU_DRAM_BYTES_PER_ELEM[n]
+        kernels[n] = {"avg_ms": kern_ms[n], "algorithmic_bytes": alg_bytes[n], "achieved_gbs": gbs,
+                      "frac_of_%s_hbm" % peak_kind: gbs / peak, "frac_of_8TBs": gbs / 8000.0,
+                      "share_of_step": kern_ms[n] / (elapsed_ms / K),
+                      "traffic": None if per_elem is None else per_elem * units[n]}
+    kernels["local_step"]["mean_steps_per_device"] = mean_steps
+    kernels["local_step"]["gelem_steps_per_s"] = N * P * mean_steps / (kern_ms["local_step"] * 1e-3) / 1e9
+    dominant = max(names, key=lambda n: kern_ms[n])
+    roofline = {"kernel": dominant, "bound": "hbm", "achieved": kernels[dominant]["achieved_gbs"],
+                "peak": peak, "unit": "GB/s", "frac": kernels[dominant]["achieved_gbs"] / peak,
+                "peak_source": "of measured (copy bandwidth of this pool's B200s)"
+                if peak_kind == "measured" else "of fallback (6650 GB/s)",
+                "traffic": kernels[dominant]["traffic"]}
+    if dominant == "local_step":
+        roofline["note"] = ("bytes per launch do not depend on the step count; at a mean of %.2f "
+                            "steps per device the kernel is limited by generator arithmetic "
+                            "(integer multiply + special-function units), not by HBM" % mean_steps)
+
+    # ---- end to end: host buffers, results read back every round -----------------------------
+    Ke = max(3, min(K, 200))
+    host_model = torch.empty(P, dtype=torch.float32).pin_memory()
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        sel = arena.run_round(r + i)
+        n2, d2 = h.stats_read()
+        h.read_params(int(sel[0]), out=host_model)
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0, world)
+    r += Ke
+    h2d = 4 * N + 4 * N + 4 * k + 4            # ids, step counts, selected ids, lr (launch parameters)
+    d2h = 2 * N * 4 + P * 4                    # statistics + the aggregated model
+    e2e = {"value": world * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": Ke,
+           "what": "round + hadfl_stats_read + hadfl_read_params(selected[0]) into pinned host memory"}
+
+    line = {"metric": METRIC, "value": world * K / (elapsed_ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": K, "warmup": warmup,
+            "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": describe(wl),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "kernels": kernels}
+
+    arena.close()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        times, what = time_oracle(wl, 1.0 / 4.0, 3)
+        line["cpu_baseline"] = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": 1,
+                                "kind": "oracle", "sample": what}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = workloads.by_name(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
