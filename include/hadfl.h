@@ -47,6 +47,7 @@ extern "C" {
 #define HADFL_ERR_INVALID 1
 #define HADFL_ERR_CUDA 2
 #define HADFL_ERR_STATE 3
+#define HADFL_ERR_TOO_LARGE 4 /* only hadfl_stats_noalloc: the problem exceeds its fixed scratch */
 
 #define HADFL_MAX_DEVICES 32 /* largest N, and therefore largest k */
 
@@ -138,6 +139,44 @@ int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_
 int hadfl_stats_enqueue(hadfl_handle *h, int32_t ref_device);
 int hadfl_stats_read(hadfl_handle *h, float *out_norm2, float *out_div2);
 int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *out_div2);
+
+/* Statistics for callers that must not allocate device memory.  (The paper has no counterpart: this
+ * is the computation of hadfl_stats behind an entry point with a different memory contract.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a process whose whole device
+ * memory has been handed to another allocator or is budgeted to the last byte, in a latency-critical
+ * loop that cannot afford the device-wide synchronisation an allocation implies, or in a component
+ * that is simply not allowed to own device memory.  Such a caller cannot even create a handle,
+ * because hadfl_init allocates the scratch of the statistics kernel.  This entry point therefore
+ * takes no handle and calls no cudaMalloc, cudaFree or any other allocating routine: its scratch
+ * (per-block partial sums and the completion ticket) lives in a fixed array of
+ * HADFL_NOALLOC_SCRATCH_BYTES inside the library image, which every GPU that loads the library
+ * holds until the process exits.
+ *
+ *   w            DEVICE pointer, 16-byte aligned, to N rows of row_stride_elems elements
+ *                (fp32 or bf16 per dtype) on the CURRENT device; read only.
+ *   out_stats    DEVICE pointer to 2N floats on the same device: norm2[0..N) then div2[0..N),
+ *                written by the kernel; valid once work enqueued on `cuda_stream` has completed.
+ *   cuda_stream  cudaStream_t the work is enqueued on.  Asynchronous.
+ *
+ * Limits: 1 <= n_devices <= HADFL_MAX_DEVICES and 1 <= n_params <= HADFL_NOALLOC_MAX_PARAMS;
+ * anything larger returns HADFL_ERR_TOO_LARGE and enqueues nothing.  Other bad arguments (NULL or
+ * misaligned pointers, stride < n_params or not a multiple of 8, ref_device out of range) return
+ * HADFL_ERR_INVALID; a failing CUDA call returns HADFL_ERR_CUDA.
+ *
+ * The first call on each device looks up the device address of the scratch array (once per
+ * device); make that first call outside any stream capture.  All calls on a device share the one
+ * array, which still holds what the previous call left there: each call re-zeroes the ticket on
+ * the stream before its kernel, and two calls whose kernels overlap on the GPU (different streams,
+ * no ordering between them) race on the scratch and give wrong sums - order them.  The result
+ * equals hadfl_stats for the same arena bit for bit when the grids agree, and within the same
+ * 1e-5 relative bound otherwise. */
+#define HADFL_NOALLOC_MAX_BLOCKS 2048
+#define HADFL_NOALLOC_SCRATCH_BYTES (256 + 2 * 8 * HADFL_NOALLOC_MAX_BLOCKS)
+#define HADFL_NOALLOC_MAX_PARAMS (((int64_t)1 << 31) - 4)
+int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t n_params,
+                        int64_t row_stride_elems, int32_t ref_device, float *out_stats,
+                        void *cuda_stream);
 
 /* Model backup (Section "Overall Design", item 9) and checkpointing.  `count` elements starting at
  * parameter 0 of device_id; bf16 storage is widened to / rounded from fp32 (nearest even).

@@ -12,7 +12,7 @@ import numpy as np
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhadfl.so")
 
-OK, ERR_INVALID, ERR_CUDA, ERR_STATE = 0, 1, 2, 3
+OK, ERR_INVALID, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, 1, 2, 3, 4
 MAX_DEVICES = 32
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 WEIGHTS_UNIFORM, WEIGHTS_VERSION = 0, 1
@@ -66,6 +66,8 @@ SIGNATURES = {
     "hadfl_stats_enqueue": (C.c_int, [_H, C.c_int32]),
     "hadfl_stats_read": (C.c_int, [_H, _f32p, _f32p]),
     "hadfl_stats": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
+    "hadfl_stats_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
+                                      C.c_void_p, C.c_void_p]),
     "hadfl_read_params": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_read_momentum": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_write_params": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
@@ -136,6 +138,14 @@ def hadfl_predict_version(series, alpha, m=1.0):
     if rc:
         raise HadflError("hadfl_predict_version", rc)
     return out.value
+
+
+def hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems, ref_device,
+                        out_stats_ptr, stream=0):
+    """Statistics for callers that must not allocate: raw DEVICE addresses in, status code out
+    (see include/hadfl.h).  out_stats_ptr: 2N device floats, norm2 then div2.  Asynchronous."""
+    return int(lib().hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems,
+                                         ref_device, out_stats_ptr, stream or None))
 
 
 # ---- the handle --------------------------------------------------------------------------------

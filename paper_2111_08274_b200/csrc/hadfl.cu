@@ -392,6 +392,61 @@ int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *ou
   return rc != HADFL_OK ? rc : hadfl_stats_read(h, out_norm2, out_div2);
 }
 
+// ---- statistics without any allocation ---------------------------------------------------------
+// Fixed scratch in the library image: [0, 256) the completion ticket, then the per-block partial
+// sums (2 doubles per block).  In host code the array's name is only a stand-in; the address that
+// kernels can use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HADFL_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kNoallocMaxGpus = 64;
+unsigned char *g_noalloc_ptr[kNoallocMaxGpus];  // device address of the scratch, per device
+int g_noalloc_sms[kNoallocMaxGpus];
+}  // namespace
+
+int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t n_params,
+                        int64_t row_stride_elems, int32_t ref_device, float *out_stats,
+                        void *cuda_stream) {
+  if (n_devices > HADFL_MAX_DEVICES || n_params > HADFL_NOALLOC_MAX_PARAMS) return HADFL_ERR_TOO_LARGE;
+  if (!w || !out_stats || n_devices < 1 || n_params < 1) return HADFL_ERR_INVALID;
+  if (dtype != HADFL_DTYPE_FP32 && dtype != HADFL_DTYPE_BF16) return HADFL_ERR_INVALID;
+  if (row_stride_elems < n_params || row_stride_elems % 8 != 0) return HADFL_ERR_INVALID;
+  if (ref_device < 0 || ref_device >= n_devices) return HADFL_ERR_INVALID;
+  if (((uintptr_t)w & 15u) || ((uintptr_t)out_stats & 3u)) return HADFL_ERR_INVALID;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoallocMaxGpus) return HADFL_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {  // set-up, once per device, with that device current
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return HADFL_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      return HADFL_ERR_CUDA;
+    g_noalloc_sms[dev] = sms;
+    g_noalloc_ptr[dev] = (unsigned char *)p;
+  }
+  unsigned int *ticket = (unsigned int *)g_noalloc_ptr[dev];
+  double *partials = (double *)(g_noalloc_ptr[dev] + 256);
+  // Same grid rule as the handle's statistics launch, capped by what the scratch holds.
+  const int64_t groups = (n_params + 3) / 4;
+  const int64_t chunks = (groups + kThreads * kStatsU - 1) / (kThreads * kStatsU);
+  int64_t lanes = ((int64_t)g_noalloc_sms[dev] * 8 + n_devices - 1) / n_devices;
+  if (lanes > chunks) lanes = chunks;
+  if (lanes * n_devices > HADFL_NOALLOC_MAX_BLOCKS) lanes = HADFL_NOALLOC_MAX_BLOCKS / n_devices;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  // The array keeps the previous call's contents: the ticket must start at zero.
+  if (cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream) != cudaSuccess) return HADFL_ERR_CUDA;
+  const unsigned blocks = (unsigned)(lanes * n_devices);
+  if (dtype == HADFL_DTYPE_BF16)
+    k_stats<__nv_bfloat16, kStatsU><<<blocks, kThreads, 0, stream>>>(
+        (const __nv_bfloat16 *)w, row_stride_elems, n_params, n_devices, ref_device, (int)lanes,
+        partials, ticket, out_stats);
+  else
+    k_stats<float, kStatsU><<<blocks, kThreads, 0, stream>>>(
+        (const float *)w, row_stride_elems, n_params, n_devices, ref_device, (int)lanes, partials,
+        ticket, out_stats);
+  return cudaGetLastError() == cudaSuccess ? HADFL_OK : HADFL_ERR_CUDA;
+}
+
 int hadfl_read_params(hadfl_handle *h, int32_t id, float *dst, int64_t count) {
   return read_row(h, id, dst, count, false);
 }
