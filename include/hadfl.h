@@ -65,7 +65,7 @@ typedef struct hadfl_config {
   int32_t dtype;            /* HADFL_DTYPE_* */
   float momentum;           /* mu of the local update */
   float weight_decay;       /* wd of the local update */
-  float grad_std;           /* standard deviation of the synthetic gradients */
+  float grad_std;           /* standard deviation of the synthetic gradients, >= 0 */
   float init_std;           /* standard deviation of the initial model */
   uint64_t seed;            /* key of the counter-based generator */
   double version_scale;     /* versions are multiplied by this before Eq. 8 (1.0 = the paper) */

@@ -207,6 +207,7 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
     return HADFL_ERR_INVALID;
   if ((cfg->w_ptr == nullptr) != (cfg->m_ptr == nullptr)) return HADFL_ERR_INVALID;
   if (!(cfg->version_scale > 0.0)) return HADFL_ERR_INVALID;
+  if (!(cfg->grad_std >= 0.0f)) return HADFL_ERR_INVALID;
   int64_t stride = cfg->row_stride_elems;
   if (stride == 0) stride = (cfg->n_params + 31) / 32 * 32;
   if (stride < cfg->n_params || stride % 8 != 0) return HADFL_ERR_INVALID;
@@ -273,21 +274,46 @@ int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *
   if (!steps || !distinct_ids(h, device_ids, n)) return HADFL_ERR_INVALID;
   for (int j = 0; j < n; ++j)
     if (steps[j] < 0) return HADFL_ERR_INVALID;
-  LocalStepArgs a;
-  memset(&a, 0, sizeof(a));
-  a.n = n;
-  for (int j = 0; j < n; ++j) {
-    const uint64_t base = h->step_count[device_ids[j]];
-    if ((base + (uint64_t)steps[j]) >> 56) return HADFL_ERR_STATE;  // the counter's stream has 2^56 steps
-    a.row[j] = device_ids[j];
-    a.steps[j] = steps[j];
-    a.base_lo[j] = (uint32_t)base;
-    a.base_hi[j] = (uint32_t)(base >> 32);
-  }
+  for (int j = 0; j < n; ++j)
+    if ((h->step_count[device_ids[j]] + (uint64_t)steps[j]) >> 56)
+      return HADFL_ERR_STATE;  // a device's gradient stream has 2^56 steps
   DeviceGuard guard(h->device);
-  const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_local_step<__nv_bfloat16>(h, a, lr)
-                                                  : launch_local_step<float>(h, a, lr);
-  if (rc != HADFL_OK) return rc;
+  // One launch covers every listed device.  A second one is needed only when some device's step
+  // counter crosses a multiple of 2^32 inside this call (once in 4 billion steps): the kernel
+  // takes the high word of the step index as fixed per launch.
+  int done[kMaxDevices];
+  for (int j = 0; j < n; ++j) done[j] = 0;
+  for (;;) {
+    LocalStepArgs a;
+    memset(&a, 0, sizeof(a));
+    bool more = false;
+    for (int j = 0; j < n; ++j) {
+      const int dev = device_ids[j];
+      const uint64_t base = h->step_count[dev] + (uint64_t)done[j];
+      const uint64_t room = ((uint64_t)1 << 32) - (base & 0xFFFFFFFFull);
+      int take = steps[j] - done[j];
+      if ((uint64_t)take > room) {
+        take = (int)room;
+        more = true;
+      }
+      if (take == 0 && done[j] > 0) continue;  // finished in an earlier launch
+      const uint64_t dp = (uint64_t)kPhiloxM1 * (uint32_t)dev;
+      const int s = a.n++;
+      a.row[s] = dev;
+      a.steps[s] = take;
+      a.base_lo[s] = (uint32_t)base;
+      a.r1_c0[s] = (uint32_t)(dp >> 32) ^ h->keys.a[0];
+      a.r1_c1[s] = (uint32_t)dp;
+      a.r1_c2[s] = (kTagGrad | ((uint32_t)(base >> 32) & 0xFFFFFFu)) ^ h->keys.b[0];
+      done[j] += take;
+    }
+    if (a.n > 0) {
+      const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_local_step<__nv_bfloat16>(h, a, lr)
+                                                      : launch_local_step<float>(h, a, lr);
+      if (rc != HADFL_OK) return rc;
+    }
+    if (!more) break;
+  }
   for (int j = 0; j < n; ++j) {
     h->step_count[device_ids[j]] += (uint64_t)steps[j];
     h->version[device_ids[j]] += (uint32_t)steps[j];

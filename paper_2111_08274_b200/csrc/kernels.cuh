@@ -119,23 +119,29 @@ __device__ __forceinline__ float sfu_cos(float x) {
   return y;
 }
 
+// -2 ln(1 - t) by its series, for t = 1 - u0 = (~x0 + 0.5) 2^-32 < 2^-10, times `scale2`:
+// 2t + t^2 + (2/3) t^3 (the next term, t^4/2, is below 2^-31 relative).  Kept out of line so that
+// the common path pays one compare and an untaken branch for it.
+__device__ __noinline__ float r2_next_to_one(uint32_t x0, float scale2) {
+  const float t = fmaf(__uint2float_rn(~x0), 0x1p-32f, 0x1p-33f);
+  return scale2 * (t * fmaf(t, fmaf(t, 0.66666667f, 1.0f), 2.0f));
+}
+
 struct NormalsFast {
-  // r^2 = -2 ln u0 = -2 ln2 * lg2(u0), except next to u0 = 1 where lg2.approx only has an absolute
-  // error bound: for x0 >= 2^32 - 2^24 (u0 > 1 - 2^-8) the exact complement t = 1 - u0 =
-  // (~x0 + 0.5) 2^-32 and the series -2 ln(1 - t) = 2t + t^2 + (2/3) t^3 (+ t^4/2 < 2^-26 relative)
-  // are used instead.  Measured against a double-precision evaluation: max |dz| about 1.5e-6.
-  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float &z0, float &z1) {
-    float r2;
-    if (x0 >= 0xFF000000u) {
-      const float t = fmaf(__uint2float_rn(~x0), 0x1p-32f, 0x1p-33f);
-      r2 = t * fmaf(t, fmaf(t, 0.66666667f, 1.0f), 2.0f);
-    } else {
-      const float u0 = fmaf(__uint2float_rn(x0), 0x1p-32f, 0x1p-33f);
-      r2 = -1.3862943611198906f * sfu_lg2(u0);
-    }
-    const float a = fmaf(__int2float_rn((int)x1), 0x1p-32f, 0x1p-33f);
+  // Two normals of standard deviation s from two words; the caller passes lg_scale = -2 ln2 s^2
+  // and scale2 = s^2 so that the scaling costs no instruction:
+  //   r^2 = lg_scale * lg2(u0)            (u0 = (x0 + 0.5) 2^-32)
+  //   theta = 2 pi a,  a = ((int)x1 + 0.5) 2^-32          (one fused multiply-add)
+  // Next to u0 = 1 (x0 >= 2^32 - 2^22) lg2.approx only has an absolute error bound, so the exact
+  // complement and a series take over.  Measured against a double-precision evaluation (s = 1):
+  // max |dz| about 2e-6, mean 1.6e-7.
+  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float lg_scale,
+                                              float scale2, float &z0, float &z1) {
+    const float u0 = fmaf(__uint2float_rn(x0), 0x1p-32f, 0x1p-33f);
+    float r2 = lg_scale * sfu_lg2(u0);
+    if (x0 >= 0xFFC00000u) r2 = r2_next_to_one(x0, scale2);
+    const float theta = fmaf(__int2float_rn((int)x1), 1.4629180792671596e-9f, 7.314590396335798e-10f);
     const float r = sfu_sqrt(r2);
-    const float theta = 6.283185307179586f * a;
     z0 = r * sfu_cos(theta);
     z1 = r * sfu_sin(theta);
   }
@@ -144,7 +150,9 @@ struct NormalsFast {
 struct NormalsAccurate {
   // Full-precision fp32 library functions; the logarithm of u0 >= 1/2 is taken through the exact
   // complement 1 - u0 = (~x0 + 0.5) 2^-32 so that it keeps its relative accuracy next to 1.
-  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float &z0, float &z1) {
+  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float lg_scale,
+                                              float scale2, float &z0, float &z1) {
+    (void)lg_scale;
     float neg_ln;
     if (x0 & 0x80000000u) {
       const float t = fmaf(__uint2float_rn(~x0), 0x1p-32f, 0x1p-33f);
@@ -154,7 +162,7 @@ struct NormalsAccurate {
       neg_ln = -logf(u0);
     }
     const float a = fmaf(__int2float_rn((int)x1), 0x1p-32f, 0x1p-33f);
-    const float r = sqrtf(2.0f * neg_ln);
+    const float r = sqrtf(2.0f * scale2 * neg_ln);
     float s, c;
     sincospif(2.0f * a, &s, &c);
     z0 = r * c;
@@ -162,13 +170,16 @@ struct NormalsAccurate {
   }
 };
 
+constexpr float kMinusTwoLn2 = -1.3862943611198906f;
+
+// Unit normals of one Philox block.
 template <typename Gen>
 __device__ __forceinline__ float4 normals_of_block(uint32_t c0, uint32_t c1, uint32_t c2,
                                                    uint32_t c3, const PhiloxKeys &keys) {
   philox4x32_10(c0, c1, c2, c3, keys);
   float4 z;
-  Gen::pair(c0, c1, z.x, z.y);
-  Gen::pair(c2, c3, z.z, z.w);
+  Gen::pair(c0, c1, kMinusTwoLn2, 1.0f, z.x, z.y);
+  Gen::pair(c2, c3, kMinusTwoLn2, 1.0f, z.z, z.w);
   return z;
 }
 
@@ -203,29 +214,43 @@ k_init(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_para
 // counts, one launch.  Thread = column group; it visits the listed rows one after the other:
 // load w and m once, run that device's steps in registers (gradient from the counter-based
 // generator), store once.  The next row's loads are issued before the current row's arithmetic.
+// The gradient noise grad_std * z is produced directly (the scale is folded into the constants
+// of the radius), which differs from rounding z first by about one part in 10^7.
 // ------------------------------------------------------------------------------------------
+// The first Philox round of a gradient block multiplies the column-group index (fixed per thread)
+// and the device id (fixed per row), so it is hoisted: the host folds the device product, the tag
+// word and the first round keys into three words per row, the thread keeps the group product, and
+// per step the round is two xors.  The host also guarantees that a row's step counter does not
+// cross a multiple of 2^32 inside one launch (it splits the call), so the step index is one add.
 struct LocalStepArgs {
   int32_t n;
   int32_t row[kMaxDevices];
   int32_t steps[kMaxDevices];
-  uint32_t base_lo[kMaxDevices];  // the device's step counter before this call
-  uint32_t base_hi[kMaxDevices];
+  uint32_t base_lo[kMaxDevices];  // low word of the device's step counter before this call
+  uint32_t r1_c0[kMaxDevices];    // hi(M1 * device) ^ key_a[0]      (xor step index -> word 0)
+  uint32_t r1_c1[kMaxDevices];    // lo(M1 * device)                                 (word 1)
+  uint32_t r1_c2[kMaxDevices];    // (tag | step_hi) ^ key_b[0]   (xor hi(M0 * group) -> word 2)
 };
 
 template <typename Gen>
-__device__ __forceinline__ void sgd_steps(float4 &w, float4 &m, uint32_t group, uint32_t device,
-                                          uint64_t base, int steps, const PhiloxKeys &keys,
-                                          float lr, float mu, float wd, float gstd) {
-  const float neg_lr = -lr;
+__device__ __forceinline__ void sgd_steps(float4 &w, float4 &m, uint32_t g_hi, uint32_t g_lo,
+                                          uint32_t r1_c0, uint32_t r1_c1, uint32_t r1_c2,
+                                          uint32_t base_lo, int steps, const PhiloxKeys &keys,
+                                          float neg_lr, float mu, float wd, float lg_scale,
+                                          float scale2) {
+  const uint32_t c2_first = g_hi ^ r1_c2;
   for (int e = 0; e < steps; ++e) {
-    const uint64_t s = base + (uint64_t)e;
-    const float4 z = normals_of_block<Gen>(group, (uint32_t)s, device,
-                                           kTagGrad | ((uint32_t)(s >> 32) & 0xFFFFFFu), keys);
+    uint32_t c0 = r1_c0 ^ (base_lo + (uint32_t)e), c1 = r1_c1, c2 = c2_first, c3 = g_lo;
+#pragma unroll
+    for (int r = 1; r < 10; ++r) philox_round(c0, c1, c2, c3, keys.a[r], keys.b[r]);
+    float4 n;  // grad_std * z
+    Gen::pair(c0, c1, lg_scale, scale2, n.x, n.y);
+    Gen::pair(c2, c3, lg_scale, scale2, n.z, n.w);
     float g;
-    g = fmaf(wd, w.x, __fmul_rn(gstd, z.x)); m.x = fmaf(mu, m.x, g); w.x = fmaf(neg_lr, m.x, w.x);
-    g = fmaf(wd, w.y, __fmul_rn(gstd, z.y)); m.y = fmaf(mu, m.y, g); w.y = fmaf(neg_lr, m.y, w.y);
-    g = fmaf(wd, w.z, __fmul_rn(gstd, z.z)); m.z = fmaf(mu, m.z, g); w.z = fmaf(neg_lr, m.z, w.z);
-    g = fmaf(wd, w.w, __fmul_rn(gstd, z.w)); m.w = fmaf(mu, m.w, g); w.w = fmaf(neg_lr, m.w, w.w);
+    g = fmaf(wd, w.x, n.x); m.x = fmaf(mu, m.x, g); w.x = fmaf(neg_lr, m.x, w.x);
+    g = fmaf(wd, w.y, n.y); m.y = fmaf(mu, m.y, g); w.y = fmaf(neg_lr, m.y, w.y);
+    g = fmaf(wd, w.z, n.z); m.z = fmaf(mu, m.z, g); w.z = fmaf(neg_lr, m.z, w.z);
+    g = fmaf(wd, w.w, n.w); m.w = fmaf(mu, m.w, g); w.w = fmaf(neg_lr, m.w, w.w);
   }
 }
 
@@ -237,6 +262,9 @@ k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t 
   const int64_t left = n_params - 4 * g;
   if (left <= 0) return;
   const int live = left >= 4 ? 4 : (int)left;
+  const unsigned long long gp = (unsigned long long)kPhiloxM0 * (uint32_t)g;
+  const uint32_t g_hi = (uint32_t)(gp >> 32), g_lo = (uint32_t)gp;
+  const float scale2 = gstd * gstd, lg_scale = kMinusTwoLn2 * scale2, neg_lr = -lr;
 
   float4 wv = ld_any(w + (int64_t)a.row[0] * stride, g, live);
   float4 mv = ld_any(m + (int64_t)a.row[0] * stride, g, live);
@@ -248,8 +276,8 @@ k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t 
     }
     const int steps = a.steps[j];
     if (steps > 0) {
-      const uint64_t base = ((uint64_t)a.base_hi[j] << 32) | a.base_lo[j];
-      sgd_steps<Gen>(wv, mv, (uint32_t)g, (uint32_t)a.row[j], base, steps, keys, lr, mu, wd, gstd);
+      sgd_steps<Gen>(wv, mv, g_hi, g_lo, a.r1_c0[j], a.r1_c1[j], a.r1_c2[j], a.base_lo[j], steps,
+                     keys, neg_lr, mu, wd, lg_scale, scale2);
       st_any(w + (int64_t)a.row[j] * stride, g, live, wv);
       st_any(m + (int64_t)a.row[j] * stride, g, live, mv);
     }
