@@ -132,6 +132,26 @@ int hadfl_aggregation_weights(hadfl_handle *h, const int32_t *selected, int32_t 
  * which also take its version.  One kernel: one read and n writes per element.  Asynchronous. */
 int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n);
 
+/* One whole round in ONE kernel: Algorithm 1's local steps of every listed device (Eq. 3), the
+ * selection (Eq. 8), the partial aggregation with write-back (Eq. 5), optionally the global
+ * synchronisation (Algorithm 1, "send w to devices whose Flag = 0": sync_all != 0 sends the
+ * aggregate to every other device) and the statistics with the aggregate as reference.  It is
+ * exactly the sequence
+ *     hadfl_local_step(device_ids, steps, n, lr); hadfl_select(round, versions, seed, k);
+ *     hadfl_aggregate(selected, k, versions); [hadfl_broadcast(selected[0], all others);]
+ *     hadfl_stats_enqueue(selected[0])
+ * - same parameters, momentum, versions and step counters, bit for bit - but each parameter and
+ * momentum value is read and written once: the aggregate is formed in registers from the freshly
+ * updated replicas and never re-read.  This is possible because selection depends on versions only,
+ * and the versions after the local steps are known before they run (versions == NULL uses them;
+ * a caller-supplied array is used as given).  The statistics are summed in a different (equally
+ * fixed) order than hadfl_stats_enqueue does, so they agree with it to rounding, not bit for bit;
+ * read them with hadfl_stats_read.  out_selected: k ids in draw order.  Devices not listed run no
+ * steps.  Asynchronous. */
+int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
+                int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
+                int32_t *out_selected);
+
 /* Per-replica statistics (not in the paper; diagnostics of how far the replicas have drifted):
  * out_norm2[i] = sum_p w_i[p]^2, out_div2[i] = sum_p (w_i[p] - w_ref[p])^2, N floats each.
  * Deterministic: fixed grid, fixed summation order, fp32 within a chunk, fp64 above.

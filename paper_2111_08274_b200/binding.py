@@ -63,6 +63,8 @@ SIGNATURES = {
     "hadfl_aggregate": (C.c_int, [_H, _i32p, C.c_int32, _f64p]),
     "hadfl_aggregation_weights": (C.c_int, [_H, _i32p, C.c_int32, _f64p, _f32p]),
     "hadfl_broadcast": (C.c_int, [_H, C.c_int32, _i32p, C.c_int32]),
+    "hadfl_round": (C.c_int, [_H, _i32p, _i32p, C.c_int32, C.c_float, C.c_int64, _f64p, C.c_uint64, C.c_int32,
+                              C.c_int32, _i32p]),
     "hadfl_stats_enqueue": (C.c_int, [_H, C.c_int32]),
     "hadfl_stats_read": (C.c_int, [_H, _f32p, _f32p]),
     "hadfl_stats": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
@@ -232,6 +234,16 @@ class Hadfl:
         dst = _arr(dst_ids, np.int32)
         self._check(self._lib.hadfl_broadcast(self._h, src, _p(dst, C.c_int32), len(dst)),
                     "hadfl_broadcast")
+
+    def round(self, device_ids, steps, lr, round_, k, seed, versions=None, sync_all=False):
+        ids, st, v = _arr(device_ids, np.int32), _arr(steps, np.int32), _arr(versions, np.float64)
+        if len(ids) != len(st):
+            raise HadflError("hadfl_round", ERR_INVALID)
+        out = np.empty(max(int(k), 1), dtype=np.int32)
+        self._check(self._lib.hadfl_round(self._h, _p(ids, C.c_int32), _p(st, C.c_int32), len(ids), lr,
+                                          round_, _p(v, C.c_double), seed, k, 1 if sync_all else 0,
+                                          _p(out, C.c_int32)), "hadfl_round")
+        return out[:k]
 
     def stats_enqueue(self, ref_device):
         self._check(self._lib.hadfl_stats_enqueue(self._h, ref_device), "hadfl_stats_enqueue")

@@ -34,13 +34,37 @@ struct hadfl_handle {
   float *d_stats = nullptr;
   int stats_lanes = 0;  // blocks per row of the statistics kernel
   bool stats_valid = false;
+  // fused round kernel scratch
+  double *d_round_partials = nullptr;
+  unsigned int *d_round_ticket = nullptr;
+  int round_grid = 0;
   int last_cuda_error = 0;
   uint64_t launches = 0;
 };
 
 namespace {
 
-constexpr int kStatsU = 4;  // column groups per thread and chunk in the statistics kernel
+constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
+
+// Columns per thread in the local-update and fused-round kernels: one Philox block for fp32
+// storage, two (one 16-byte access of w) for bf16 storage.
+template <typename WT>
+struct StepPack {
+  static constexpr int E = Pack16<WT>::E;
+};
+
+// What the kernels need to know about one device's steps in one launch.
+RowStep row_step(const hadfl_handle *h, int dev, uint64_t base, int steps) {
+  const uint64_t dp = (uint64_t)kPhiloxM1 * (uint32_t)dev;
+  RowStep r;
+  r.row = dev;
+  r.steps = steps;
+  r.base_lo = (uint32_t)base;
+  r.r1_c0 = (uint32_t)(dp >> 32) ^ h->keys.a[0];
+  r.r1_c1 = (uint32_t)dp;
+  r.r1_c2 = (kTagGrad | ((uint32_t)(base >> 32) & 0xFFFFFFu)) ^ h->keys.b[0];
+  return r;
+}
 
 #define HADFL_CUDA(h, expr)                       \
   do {                                            \
@@ -64,8 +88,6 @@ struct DeviceGuard {
 };
 
 inline size_t elem_size(const hadfl_handle *h) { return h->cfg.dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
-
-inline int64_t n_groups(const hadfl_handle *h) { return (h->cfg.n_params + 3) / 4; }
 
 bool distinct_ids(const hadfl_handle *h, const int32_t *ids, int n) {
   if (!ids || n < 1 || n > h->cfg.n_devices) return false;
@@ -100,17 +122,37 @@ int launch_init(hadfl_handle *h) {
 
 template <typename WT>
 int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
-  const unsigned blocks = (unsigned)((n_groups(h) + kThreads - 1) / kThreads);
-  k_local_step<WT, NormalsFast><<<blocks, kThreads, 0, h->stream>>>(
+  constexpr int E = StepPack<WT>::E;
+  const int64_t packs = (h->cfg.n_params + E - 1) / E;
+  const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
+  k_local_step<WT, NormalsFast, E><<<blocks, kThreads, 0, h->stream>>>(
       (WT *)h->w, h->m, h->stride, h->cfg.n_params, a, h->keys, lr, h->cfg.momentum,
       h->cfg.weight_decay, h->cfg.grad_std);
   return check_launch(h);
 }
 
+template <typename WT>
+int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
+  k_round<WT, NormalsFast, StepPack<WT>::E><<<h->round_grid, kThreads, 0, h->stream>>>(
+      (WT *)h->w, h->m, h->stride, h->cfg.n_params, a, h->keys, lr, h->cfg.momentum,
+      h->cfg.weight_decay, h->cfg.grad_std, h->d_round_partials, h->d_round_ticket, h->d_stats);
+  return check_launch(h);
+}
+
+template <typename WT>
+int round_blocks_per_sm() {
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+          &n, k_round<WT, NormalsFast, StepPack<WT>::E>, kThreads, 0) != cudaSuccess || n < 1)
+    n = 1;
+  return n;
+}
+
 template <typename WT, int KR, int U>
 int launch_combine_as(hadfl_handle *h, const CombineArgs &c) {
-  const int64_t per_block = (int64_t)kThreads * U;
-  const unsigned blocks = (unsigned)((n_groups(h) + per_block - 1) / per_block);
+  constexpr int E = Pack16<WT>::E;
+  const int64_t per_block = (int64_t)kThreads * U * E;
+  const unsigned blocks = (unsigned)((h->cfg.n_params + per_block - 1) / per_block);
   k_combine<WT, KR, U><<<blocks, kThreads, 0, h->stream>>>((WT *)h->w, h->stride,
                                                             h->cfg.n_params, c);
   return check_launch(h);
@@ -240,7 +282,9 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   }
   // Statistics grid: one wave of resident blocks (8 blocks of 256 threads per SM), split evenly
   // over the rows; never more blocks per row than there are column chunks.
-  const int64_t chunks = (n_groups(h) + kThreads * kStatsU - 1) / (kThreads * kStatsU);
+  const int64_t pack_e = cfg->dtype == HADFL_DTYPE_BF16 ? 8 : 4;
+  const int64_t packs = (cfg->n_params + pack_e - 1) / pack_e;
+  const int64_t chunks = (packs + kThreads * kStatsU - 1) / (kThreads * kStatsU);
   int64_t lanes = ((int64_t)h->sm_count * 8 + cfg->n_devices - 1) / cfg->n_devices;
   if (lanes > chunks) lanes = chunks;
   h->stats_lanes = (int)lanes;
@@ -248,6 +292,19 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
                            sizeof(double) * 2 * (size_t)cfg->n_devices * (size_t)lanes));
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_ticket, sizeof(unsigned int)));
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
+  // Fused round kernel: one resident wave, never more blocks than there are packs to visit.
+  {
+    const int per_sm = cfg->dtype == HADFL_DTYPE_BF16 ? round_blocks_per_sm<__nv_bfloat16>()
+                                                      : round_blocks_per_sm<float>();
+    int64_t grid = (int64_t)h->sm_count * per_sm;
+    const int64_t need = (packs + kThreads - 1) / kThreads;
+    if (grid > need) grid = need;
+    h->round_grid = (int)grid;
+  }
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_partials,
+                           sizeof(double) * 2 * kMaxDevices * (size_t)h->round_grid));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_ticket, sizeof(unsigned int)));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
   return cfg->dtype == HADFL_DTYPE_BF16 ? launch_init<__nv_bfloat16>(h) : launch_init<float>(h);
@@ -264,6 +321,8 @@ int hadfl_destroy(hadfl_handle *h) {
   cudaFree(h->d_partials);
   cudaFree(h->d_ticket);
   cudaFree(h->d_stats);
+  cudaFree(h->d_round_partials);
+  cudaFree(h->d_round_ticket);
   delete h;
   return HADFL_OK;
 }
@@ -297,14 +356,7 @@ int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *
         more = true;
       }
       if (take == 0 && done[j] > 0) continue;  // finished in an earlier launch
-      const uint64_t dp = (uint64_t)kPhiloxM1 * (uint32_t)dev;
-      const int s = a.n++;
-      a.row[s] = dev;
-      a.steps[s] = take;
-      a.base_lo[s] = (uint32_t)base;
-      a.r1_c0[s] = (uint32_t)(dp >> 32) ^ h->keys.a[0];
-      a.r1_c1[s] = (uint32_t)dp;
-      a.r1_c2[s] = (kTagGrad | ((uint32_t)(base >> 32) & 0xFFFFFFu)) ^ h->keys.b[0];
+      a.r[a.n++] = row_step(h, dev, base, take);
       done[j] += take;
     }
     if (a.n > 0) {
@@ -389,6 +441,84 @@ int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_
   return HADFL_OK;
 }
 
+int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
+                int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
+                int32_t *out_selected) {
+  if (!h || !out_selected) return HADFL_ERR_INVALID;
+  if (!steps || !distinct_ids(h, device_ids, n)) return HADFL_ERR_INVALID;
+  const int N = h->cfg.n_devices;
+  int row_steps[kMaxDevices];
+  for (int i = 0; i < N; ++i) row_steps[i] = 0;
+  bool crosses = false;
+  for (int j = 0; j < n; ++j) {
+    if (steps[j] < 0) return HADFL_ERR_INVALID;
+    const uint64_t base = h->step_count[device_ids[j]];
+    if ((base + (uint64_t)steps[j]) >> 56) return HADFL_ERR_STATE;
+    if ((base & 0xFFFFFFFFull) + (uint64_t)steps[j] > ((uint64_t)1 << 32)) crosses = true;
+    row_steps[device_ids[j]] = steps[j];
+  }
+  // Selection sees the versions as they will be after the local steps.
+  double x[kMaxDevices];
+  for (int i = 0; i < N; ++i)
+    x[i] = (versions ? versions[i] : (double)(h->version[i] + (uint32_t)row_steps[i])) *
+           h->cfg.version_scale;
+  int32_t sel[kMaxDevices];
+  if (!selection_draw(x, h->avail, N, round, seed, k, sel)) return HADFL_ERR_INVALID;
+
+  if (crosses) {
+    // A step counter crosses a multiple of 2^32 in this call (once in 4 billion steps): take the
+    // separate kernels, which split the launch.
+    int rc = hadfl_local_step(h, device_ids, steps, n, lr);
+    if (rc == HADFL_OK) rc = hadfl_aggregate(h, sel, k, versions);
+    if (rc == HADFL_OK && sync_all) {
+      int32_t others[kMaxDevices];
+      int n_others = 0;
+      uint32_t in_sel = 0;
+      for (int j = 0; j < k; ++j) in_sel |= 1u << sel[j];
+      for (int i = 0; i < N; ++i)
+        if (!(in_sel & (1u << i))) others[n_others++] = i;
+      rc = hadfl_broadcast(h, sel[0], others, n_others);
+    }
+    if (rc == HADFL_OK) rc = hadfl_stats_enqueue(h, sel[0]);
+    if (rc != HADFL_OK) return rc;
+    for (int j = 0; j < k; ++j) out_selected[j] = sel[j];
+    return HADFL_OK;
+  }
+
+  RoundArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = N;
+  a.k = k;
+  a.write_all = sync_all ? 1 : 0;
+  aggregation_weights(h->cfg.weight_mode, x, h->avail, N, sel, k, a.a);
+  uint32_t in_sel = 0;
+  int pos = 0;
+  for (int j = 0; j < k; ++j) {
+    a.r[pos++] = row_step(h, sel[j], h->step_count[sel[j]], row_steps[sel[j]]);
+    in_sel |= 1u << sel[j];
+  }
+  for (int i = 0; i < N; ++i)
+    if (!(in_sel & (1u << i))) a.r[pos++] = row_step(h, i, h->step_count[i], row_steps[i]);
+  {
+    DeviceGuard guard(h->device);
+    const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_round<__nv_bfloat16>(h, a, lr)
+                                                    : launch_round<float>(h, a, lr);
+    if (rc != HADFL_OK) return rc;
+  }
+  for (int i = 0; i < N; ++i) {
+    h->step_count[i] += (uint64_t)row_steps[i];
+    h->version[i] += (uint32_t)row_steps[i];
+  }
+  uint32_t vmax = 0;
+  for (int j = 0; j < k; ++j) vmax = h->version[sel[j]] > vmax ? h->version[sel[j]] : vmax;
+  for (int j = 0; j < k; ++j) h->version[sel[j]] = vmax;
+  if (sync_all)
+    for (int i = 0; i < N; ++i) h->version[i] = vmax;
+  h->stats_valid = true;
+  for (int j = 0; j < k; ++j) out_selected[j] = sel[j];
+  return HADFL_OK;
+}
+
 int hadfl_stats_enqueue(hadfl_handle *h, int32_t ref_device) {
   if (!h || ref_device < 0 || ref_device >= h->cfg.n_devices) return HADFL_ERR_INVALID;
   DeviceGuard guard(h->device);
@@ -453,8 +583,9 @@ int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t
   unsigned int *ticket = (unsigned int *)g_noalloc_ptr[dev];
   double *partials = (double *)(g_noalloc_ptr[dev] + 256);
   // Same grid rule as the handle's statistics launch, capped by what the scratch holds.
-  const int64_t groups = (n_params + 3) / 4;
-  const int64_t chunks = (groups + kThreads * kStatsU - 1) / (kThreads * kStatsU);
+  const int64_t pack_e = dtype == HADFL_DTYPE_BF16 ? 8 : 4;
+  const int64_t packs = (n_params + pack_e - 1) / pack_e;
+  const int64_t chunks = (packs + kThreads * kStatsU - 1) / (kThreads * kStatsU);
   int64_t lanes = ((int64_t)g_noalloc_sms[dev] * 8 + n_devices - 1) / n_devices;
   if (lanes > chunks) lanes = chunks;
   if (lanes * n_devices > HADFL_NOALLOC_MAX_BLOCKS) lanes = HADFL_NOALLOC_MAX_BLOCKS / n_devices;

@@ -89,6 +89,98 @@ __device__ __forceinline__ void st_any(T *row, int64_t g, int live, float4 v) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Packs: E consecutive parameters held by one thread (E = 4 or 8).  fp32: E/4 128-bit accesses;
+// bf16: one 64-bit (E = 4) or 128-bit (E = 8) access.  A pack of 8 is two column groups, i.e.
+// two Philox blocks.  `live` < E only in the ragged last pack of a row.
+// ------------------------------------------------------------------------------------------
+template <typename WT>
+struct Pack16 {  // the pack that is 16 bytes of storage
+  static constexpr int E = sizeof(WT) == 2 ? 8 : 4;
+};
+
+template <int E>
+__device__ __forceinline__ void ld_pack(const float *row, int64_t p, float (&v)[E]) {
+#pragma unroll
+  for (int i = 0; i < E / 4; ++i) {
+    const float4 t = *reinterpret_cast<const float4 *>(row + E * p + 4 * i);
+    v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
+  }
+}
+template <int E>
+__device__ __forceinline__ void st_pack(float *row, int64_t p, const float (&v)[E]) {
+#pragma unroll
+  for (int i = 0; i < E / 4; ++i)
+    *reinterpret_cast<float4 *>(row + E * p + 4 * i) =
+        make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+__device__ __forceinline__ void bf16x2_to_floats(uint32_t raw, float &lo, float &hi) {
+  lo = __uint_as_float(raw << 16);
+  hi = __uint_as_float(raw & 0xFFFF0000u);
+}
+__device__ __forceinline__ uint32_t floats_to_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&t);
+}
+template <int E>
+__device__ __forceinline__ void ld_pack(const __nv_bfloat16 *row, int64_t p, float (&v)[E]) {
+  if (E == 8) {
+    const uint4 raw = *reinterpret_cast<const uint4 *>(row + 8 * p);
+    bf16x2_to_floats(raw.x, v[0], v[1]);
+    bf16x2_to_floats(raw.y, v[2], v[3]);
+    bf16x2_to_floats(raw.z, v[E - 4], v[E - 3]);
+    bf16x2_to_floats(raw.w, v[E - 2], v[E - 1]);
+  } else {
+    const uint2 raw = *reinterpret_cast<const uint2 *>(row + 4 * p);
+    bf16x2_to_floats(raw.x, v[0], v[1]);
+    bf16x2_to_floats(raw.y, v[2], v[3]);
+  }
+}
+template <int E>
+__device__ __forceinline__ void st_pack(__nv_bfloat16 *row, int64_t p, const float (&v)[E]) {
+  if (E == 8) {
+    uint4 raw;
+    raw.x = floats_to_bf16x2(v[0], v[1]);
+    raw.y = floats_to_bf16x2(v[2], v[3]);
+    raw.z = floats_to_bf16x2(v[E - 4], v[E - 3]);
+    raw.w = floats_to_bf16x2(v[E - 2], v[E - 1]);
+    *reinterpret_cast<uint4 *>(row + 8 * p) = raw;
+  } else {
+    uint2 raw;
+    raw.x = floats_to_bf16x2(v[0], v[1]);
+    raw.y = floats_to_bf16x2(v[2], v[3]);
+    *reinterpret_cast<uint2 *>(row + 4 * p) = raw;
+  }
+}
+template <typename T, int E>
+__device__ __forceinline__ void ld_pack_any(const T *row, int64_t p, int live, float (&v)[E]) {
+  if (live == E) {
+    ld_pack<E>(row, p, v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < E; ++i) v[i] = i < live ? ld_elem(row, E * p + i) : 0.f;
+  }
+}
+template <typename T, int E>
+__device__ __forceinline__ void st_pack_any(T *row, int64_t p, int live, const float (&v)[E]) {
+  if (live == E) {
+    st_pack<E>(row, p, v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < E; ++i)
+      if (i < live) st_elem(row, E * p + i, v[i]);
+  }
+}
+// The value a parameter has once stored: itself for fp32, rounded to nearest even for bf16.
+__device__ __forceinline__ float as_stored(float v, const float *) { return v; }
+__device__ __forceinline__ float as_stored(float v, const __nv_bfloat16 *) {
+  return __bfloat162float(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ int live_of(int64_t n_params, int64_t p, int E) {
+  const int64_t left = n_params - (int64_t)E * p;
+  return left >= E ? E : (left > 0 ? (int)left : 0);
+}
+
+// ------------------------------------------------------------------------------------------
 // Uniform words -> standard normals (Box-Muller).  (x0, x1) -> (z0, z1):
 //   u0 = (x0 + 0.5) 2^-32,  u1 = (x1 + 0.5) 2^-32,  r = sqrt(-2 ln u0),
 //   z0 = r cos(2 pi u1),    z1 = r sin(2 pi u1).
@@ -211,78 +303,111 @@ k_init(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_para
 
 // ------------------------------------------------------------------------------------------
 // K1: batched local update (Eq. 3 / Algorithm 1) for a list of devices with per-device step
-// counts, one launch.  Thread = column group; it visits the listed rows one after the other:
-// load w and m once, run that device's steps in registers (gradient from the counter-based
-// generator), store once.  The next row's loads are issued before the current row's arithmetic.
-// The gradient noise grad_std * z is produced directly (the scale is folded into the constants
-// of the radius), which differs from rounding z first by about one part in 10^7.
-// ------------------------------------------------------------------------------------------
+// counts, one launch.  A thread owns a pack of E columns (E/4 Philox blocks) and visits the listed
+// rows one after the other: load w and m once, run that device's steps in registers (gradient
+// from the counter-based generator), store once.  The next row's loads are issued before the
+// current row's arithmetic.  The gradient noise grad_std * z is produced directly (the scale is
+// folded into the constants of the radius), which differs from rounding z first by about one
+// part in 10^7.
+//
 // The first Philox round of a gradient block multiplies the column-group index (fixed per thread)
 // and the device id (fixed per row), so it is hoisted: the host folds the device product, the tag
 // word and the first round keys into three words per row, the thread keeps the group product, and
 // per step the round is two xors.  The host also guarantees that a row's step counter does not
 // cross a multiple of 2^32 inside one launch (it splits the call), so the step index is one add.
-struct LocalStepArgs {
-  int32_t n;
-  int32_t row[kMaxDevices];
-  int32_t steps[kMaxDevices];
-  uint32_t base_lo[kMaxDevices];  // low word of the device's step counter before this call
-  uint32_t r1_c0[kMaxDevices];    // hi(M1 * device) ^ key_a[0]      (xor step index -> word 0)
-  uint32_t r1_c1[kMaxDevices];    // lo(M1 * device)                                 (word 1)
-  uint32_t r1_c2[kMaxDevices];    // (tag | step_hi) ^ key_b[0]   (xor hi(M0 * group) -> word 2)
+// ------------------------------------------------------------------------------------------
+struct RowStep {
+  int32_t row;
+  int32_t steps;
+  uint32_t base_lo;  // low word of the device's step counter before this call
+  uint32_t r1_c0;    // hi(M1 * device) ^ key_a[0]      (xor step index -> word 0)
+  uint32_t r1_c1;    // lo(M1 * device)                                 (word 1)
+  uint32_t r1_c2;    // (tag | step_hi) ^ key_b[0]   (xor hi(M0 * group) -> word 2)
 };
 
-template <typename Gen>
-__device__ __forceinline__ void sgd_steps(float4 &w, float4 &m, uint32_t g_hi, uint32_t g_lo,
-                                          uint32_t r1_c0, uint32_t r1_c1, uint32_t r1_c2,
-                                          uint32_t base_lo, int steps, const PhiloxKeys &keys,
-                                          float neg_lr, float mu, float wd, float lg_scale,
-                                          float scale2) {
-  const uint32_t c2_first = g_hi ^ r1_c2;
-  for (int e = 0; e < steps; ++e) {
-    uint32_t c0 = r1_c0 ^ (base_lo + (uint32_t)e), c1 = r1_c1, c2 = c2_first, c3 = g_lo;
+struct LocalStepArgs {
+  int32_t n;
+  RowStep r[kMaxDevices];
+};
+
+struct StepConsts {
+  float neg_lr, mu, wd, lg_scale, scale2;
+};
+
+// The thread's share of the first Philox round: hi/lo of M0 * group for each of its NB groups.
+template <int NB>
+struct GroupProducts {
+  uint32_t hi[NB], lo[NB];
+  __device__ __forceinline__ explicit GroupProducts(int64_t pack) {
 #pragma unroll
-    for (int r = 1; r < 10; ++r) philox_round(c0, c1, c2, c3, keys.a[r], keys.b[r]);
-    float4 n;  // grad_std * z
-    Gen::pair(c0, c1, lg_scale, scale2, n.x, n.y);
-    Gen::pair(c2, c3, lg_scale, scale2, n.z, n.w);
-    float g;
-    g = fmaf(wd, w.x, n.x); m.x = fmaf(mu, m.x, g); w.x = fmaf(neg_lr, m.x, w.x);
-    g = fmaf(wd, w.y, n.y); m.y = fmaf(mu, m.y, g); w.y = fmaf(neg_lr, m.y, w.y);
-    g = fmaf(wd, w.z, n.z); m.z = fmaf(mu, m.z, g); w.z = fmaf(neg_lr, m.z, w.z);
-    g = fmaf(wd, w.w, n.w); m.w = fmaf(mu, m.w, g); w.w = fmaf(neg_lr, m.w, w.w);
+    for (int b = 0; b < NB; ++b) {
+      const unsigned long long gp = (unsigned long long)kPhiloxM0 * (uint32_t)(pack * NB + b);
+      hi[b] = (uint32_t)(gp >> 32);
+      lo[b] = (uint32_t)gp;
+    }
+  }
+};
+
+template <typename Gen, int NB>
+__device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB],
+                                          const GroupProducts<NB> &gp, const RowStep &rs,
+                                          const PhiloxKeys &keys, const StepConsts &k) {
+  uint32_t c2_first[NB];
+#pragma unroll
+  for (int b = 0; b < NB; ++b) c2_first[b] = gp.hi[b] ^ rs.r1_c2;
+  for (int e = 0; e < rs.steps; ++e) {
+    const uint32_t c0_first = rs.r1_c0 ^ (rs.base_lo + (uint32_t)e);
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      uint32_t c0 = c0_first, c1 = rs.r1_c1, c2 = c2_first[b], c3 = gp.lo[b];
+#pragma unroll
+      for (int r = 1; r < 10; ++r) philox_round(c0, c1, c2, c3, keys.a[r], keys.b[r]);
+      float n[4];  // grad_std * z
+      Gen::pair(c0, c1, k.lg_scale, k.scale2, n[0], n[1]);
+      Gen::pair(c2, c3, k.lg_scale, k.scale2, n[2], n[3]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float g = fmaf(k.wd, w[4 * b + i], n[i]);
+        m[4 * b + i] = fmaf(k.mu, m[4 * b + i], g);
+        w[4 * b + i] = fmaf(k.neg_lr, m[4 * b + i], w[4 * b + i]);
+      }
+    }
   }
 }
 
-template <typename WT, typename Gen>
+template <typename WT, typename Gen, int E>
 __global__ void __launch_bounds__(kThreads)
 k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_params,
              LocalStepArgs a, PhiloxKeys keys, float lr, float mu, float wd, float gstd) {
-  const int64_t g = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  const int64_t left = n_params - 4 * g;
-  if (left <= 0) return;
-  const int live = left >= 4 ? 4 : (int)left;
-  const unsigned long long gp = (unsigned long long)kPhiloxM0 * (uint32_t)g;
-  const uint32_t g_hi = (uint32_t)(gp >> 32), g_lo = (uint32_t)gp;
-  const float scale2 = gstd * gstd, lg_scale = kMinusTwoLn2 * scale2, neg_lr = -lr;
+  const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int live = live_of(n_params, p, E);
+  if (live == 0) return;
+  const GroupProducts<E / 4> gp(p);
+  StepConsts k;
+  k.scale2 = gstd * gstd;
+  k.lg_scale = kMinusTwoLn2 * k.scale2;
+  k.neg_lr = -lr;
+  k.mu = mu;
+  k.wd = wd;
 
-  float4 wv = ld_any(w + (int64_t)a.row[0] * stride, g, live);
-  float4 mv = ld_any(m + (int64_t)a.row[0] * stride, g, live);
+  float wv[E], mv[E], wn[E], mn[E];
+  ld_pack_any(w + (int64_t)a.r[0].row * stride, p, live, wv);
+  ld_pack_any(m + (int64_t)a.r[0].row * stride, p, live, mv);
   for (int j = 0; j < a.n; ++j) {
-    float4 wn = wv, mn = mv;
     if (j + 1 < a.n) {
-      wn = ld_any(w + (int64_t)a.row[j + 1] * stride, g, live);
-      mn = ld_any(m + (int64_t)a.row[j + 1] * stride, g, live);
+      ld_pack_any(w + (int64_t)a.r[j + 1].row * stride, p, live, wn);
+      ld_pack_any(m + (int64_t)a.r[j + 1].row * stride, p, live, mn);
     }
-    const int steps = a.steps[j];
-    if (steps > 0) {
-      sgd_steps<Gen>(wv, mv, g_hi, g_lo, a.r1_c0[j], a.r1_c1[j], a.r1_c2[j], a.base_lo[j], steps,
-                     keys, neg_lr, mu, wd, lg_scale, scale2);
-      st_any(w + (int64_t)a.row[j] * stride, g, live, wv);
-      st_any(m + (int64_t)a.row[j] * stride, g, live, mv);
+    if (a.r[j].steps > 0) {
+      sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+      st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, wv);
+      st_pack_any(m + (int64_t)a.r[j].row * stride, p, live, mv);
     }
-    wv = wn;
-    mv = mn;
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      wv[i] = wn[i];
+      mv[i] = mn[i];
+    }
   }
 }
 
@@ -291,9 +416,9 @@ k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t 
 //   partial aggregation (Eq. 5): read list = write list = the selected devices, weights a_j;
 //   global synchronisation (Algorithm 1): read list = {source}, weight 1, write list = receivers.
 //   acc = a_0 * w[rd_0];  acc = fma(a_j, w[rd_j], acc) for j = 1 .. nr-1, in list order.
-// KR > 0: compile-time read count (all loads of a thread issued before the first multiply);
-// KR == 0: any read count, loads issued in batches of 8.  U column groups per thread keep enough
-// bytes in flight when the read list is short.
+// A thread owns U 16-byte packs.  KR > 0: compile-time read count; KR == 0: any read count.  The
+// row loads of a pack are issued in batches of B rows (B * E values in registers) before the
+// batch's multiply-adds; U packs per thread keep enough bytes in flight when the list is short.
 // ------------------------------------------------------------------------------------------
 struct CombineArgs {
   int32_t nr;
@@ -303,87 +428,60 @@ struct CombineArgs {
   int32_t wr[kMaxDevices];
 };
 
-template <typename WT, int KR>
-__device__ __forceinline__ float4 combine_group(const WT *__restrict__ w, int64_t stride,
-                                                const CombineArgs &c, int64_t g, int live) {
-  float4 acc;
-  if (KR > 0) {
-    float4 v[KR > 0 ? KR : 1];
+template <typename WT, int KR, int E>
+__device__ __forceinline__ void combine_pack(const WT *__restrict__ w, int64_t stride,
+                                             const CombineArgs &c, int64_t p, int live,
+                                             float (&acc)[E]) {
+  constexpr int B = KR > 0 ? (KR * E <= 64 ? KR : 64 / E) : 32 / E;
+  const int nr = KR > 0 ? KR : c.nr;
 #pragma unroll
-    for (int j = 0; j < KR; ++j) v[j] = ld_any(w + (int64_t)c.rd[j] * stride, g, live);
-    acc.x = __fmul_rn(c.a[0], v[0].x);
-    acc.y = __fmul_rn(c.a[0], v[0].y);
-    acc.z = __fmul_rn(c.a[0], v[0].z);
-    acc.w = __fmul_rn(c.a[0], v[0].w);
+  for (int i = 0; i < E; ++i) acc[i] = 0.f;
 #pragma unroll
-    for (int j = 1; j < KR; ++j) {
-      acc.x = fmaf(c.a[j], v[j].x, acc.x);
-      acc.y = fmaf(c.a[j], v[j].y, acc.y);
-      acc.z = fmaf(c.a[j], v[j].z, acc.z);
-      acc.w = fmaf(c.a[j], v[j].w, acc.w);
-    }
-  } else {
-    acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int base = 0; base < c.nr; base += 8) {
-      float4 v[8];
+  for (int base = 0; base < (KR > 0 ? KR : kMaxDevices); base += B) {
+    if (base >= nr) break;
+    float v[B][E];
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (base + j < c.nr) v[j] = ld_any(w + (int64_t)c.rd[base + j] * stride, g, live);
+    for (int j = 0; j < B; ++j)
+      if (base + j < nr) ld_pack_any(w + (int64_t)c.rd[base + j] * stride, p, live, v[j]);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (base + j < c.nr) {
-          const float aj = c.a[base + j];
-          if (base + j == 0) {
-            acc.x = __fmul_rn(aj, v[j].x);
-            acc.y = __fmul_rn(aj, v[j].y);
-            acc.z = __fmul_rn(aj, v[j].z);
-            acc.w = __fmul_rn(aj, v[j].w);
-          } else {
-            acc.x = fmaf(aj, v[j].x, acc.x);
-            acc.y = fmaf(aj, v[j].y, acc.y);
-            acc.z = fmaf(aj, v[j].z, acc.z);
-            acc.w = fmaf(aj, v[j].w, acc.w);
-          }
+    for (int j = 0; j < B; ++j) {
+      if (base + j < nr) {
+        const float aj = c.a[base + j];
+        if (base + j == 0) {
+#pragma unroll
+          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(aj, v[j][i]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, v[j][i], acc[i]);
         }
       }
     }
   }
-  return acc;
 }
 
 template <typename WT, int KR, int U>
 __global__ void __launch_bounds__(kThreads)
 k_combine(WT *__restrict__ w, int64_t stride, int64_t n_params, CombineArgs c) {
-  const int64_t n_groups = (n_params + 3) >> 2;
-  const int64_t g0 = (int64_t)blockIdx.x * (kThreads * U) + threadIdx.x;
-  float4 acc[U];
+  constexpr int E = Pack16<WT>::E;
+  const int64_t p0 = (int64_t)blockIdx.x * (kThreads * U) + threadIdx.x;
+  float acc[U][E];
   int live[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    const int64_t g = g0 + (int64_t)u * kThreads;
-    const int64_t left = n_params - 4 * g;
-    live[u] = g < n_groups ? (left >= 4 ? 4 : (int)left) : 0;
-    if (live[u] > 0) acc[u] = combine_group<WT, KR>(w, stride, c, g, live[u]);
+    const int64_t p = p0 + (int64_t)u * kThreads;
+    live[u] = live_of(n_params, p, E);
+    if (live[u] > 0) combine_pack<WT, KR, E>(w, stride, c, p, live[u], acc[u]);
   }
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    const int64_t g = g0 + (int64_t)u * kThreads;
+    const int64_t p = p0 + (int64_t)u * kThreads;
     if (live[u] > 0)
-      for (int j = 0; j < c.nw; ++j) st_any(w + (int64_t)c.wr[j] * stride, g, live[u], acc[u]);
+      for (int j = 0; j < c.nw; ++j) st_pack_any(w + (int64_t)c.wr[j] * stride, p, live[u], acc[u]);
   }
 }
 
 // ------------------------------------------------------------------------------------------
-// K3: per-replica squared norm and squared distance to a reference replica.
-// Block b works on row b % N and on the column chunks (b / N), (b / N) + lanes, ...; a chunk is
-// kThreads * U column groups.  Blocks that are neighbours in launch order work on the same chunk
-// of different rows at about the same time, so the reference chunk is fetched from HBM once and
-// found in L2 by the others: HBM traffic stays N * P elements.
-// Per thread: fp32 sums over the 4*U elements of a chunk in a fixed order, accumulated in fp64
-// across chunks; butterfly over the warp and a fixed-order sum over the warps (fp64) give
-// partials[which][row][lane].  The block that takes the last ticket sums the partials of each row
-// in a fixed order -> out[2N] (norm2 then div2) and resets the ticket.  No block waits for
-// another; fixed grid and fixed orders make the result reproducible bit for bit.
+// Deterministic reductions shared by the statistics kernel and the fused round kernel.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -391,49 +489,97 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
+// Sums two per-lane values over the warp with five shuffles: after the first exchange the lower
+// half-warp carries `a` and the upper half carries `b`.  Lane 0 ends with sum(a), lane 16 with
+// sum(b); the order of additions is fixed.
+__device__ __forceinline__ float warp_sum_pair(float a, float b, int lane) {
+  const bool upper = (lane & 16) != 0;
+  float mine = upper ? b : a;
+  const float give = upper ? a : b;
+  mine += __shfl_xor_sync(0xFFFFFFFFu, give, 16);
+#pragma unroll
+  for (int off = 8; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
+  return mine;
+}
+
+// Last-block finish: the block that draws the last ticket sums partials[t][0 .. n_src) for every
+// t < n_vals in a fixed order (a warp per value, lanes strided, then the butterfly), hands the
+// sums to `emit`, and resets the ticket.  Returns without waiting for anyone.
+template <typename Emit>
+__device__ __forceinline__ void finish_by_last_block(const double *__restrict__ partials,
+                                                     int n_vals, int n_src,
+                                                     unsigned int *__restrict__ ticket,
+                                                     bool *s_last, Emit emit) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) *s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!*s_last) return;
+  __threadfence();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int t = warp; t < n_vals; t += kThreads / 32) {
+    const double *src = partials + (int64_t)t * n_src;
+    double s = 0.0;
+    for (int l = lane; l < n_src; l += 32) s += __ldcg(src + l);
+    s = warp_sum(s);
+    if (lane == 0) emit(t, s);
+  }
+  if (threadIdx.x == 0) *ticket = 0u;
+}
+
+// ------------------------------------------------------------------------------------------
+// K3: per-replica squared norm and squared distance to a reference replica.
+// Block b works on row b % N and on the chunks (b / N), (b / N) + lanes, ...; a chunk is
+// kThreads * U 16-byte packs.  Blocks that are neighbours in launch order work on the same chunk
+// of different rows at about the same time, so the reference chunk is fetched from HBM once and
+// found in L2 by the others: HBM traffic stays N * P elements.
+// Per thread: fp32 sums over the elements of a chunk in a fixed order, accumulated in fp64 across
+// chunks; butterfly over the warp and a fixed-order sum over the warps (fp64) give
+// partials[which * N + row][lane].  The last-ticket block sums them -> out[2N] (norm2 then div2).
+// No block waits for another; fixed grid and fixed orders make the result reproducible.
+// ------------------------------------------------------------------------------------------
 template <typename WT, int U>
 __global__ void __launch_bounds__(kThreads)
 k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_devices, int ref,
         int lanes, double *__restrict__ partials, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
   constexpr int kWarps = kThreads / 32;
+  constexpr int E = Pack16<WT>::E;
   __shared__ double s_part[2][kWarps];
   __shared__ bool s_last;
   const int row = blockIdx.x % n_devices;
   const int my_lane = blockIdx.x / n_devices;
-  const int64_t n_groups = (n_params + 3) >> 2;
+  const int64_t n_packs = (n_params + E - 1) / E;
   const int64_t per_chunk = (int64_t)kThreads * U;
-  const int64_t n_chunks = (n_groups + per_chunk - 1) / per_chunk;
+  const int64_t n_chunks = (n_packs + per_chunk - 1) / per_chunk;
   const WT *my_row = w + (int64_t)row * stride;
   const WT *ref_row = w + (int64_t)ref * stride;
 
   double n2 = 0.0, d2 = 0.0;
   for (int64_t chunk = my_lane; chunk < n_chunks; chunk += lanes) {
-    const int64_t g0 = chunk * per_chunk + threadIdx.x;
-    float4 v[U], r[U];
+    const int64_t p0 = chunk * per_chunk + threadIdx.x;
+    float v[U][E], r[U][E];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int64_t g = g0 + (int64_t)u * kThreads;
-      const int64_t left = n_params - 4 * g;
-      if (left >= 4) {
-        v[u] = ld_group(my_row, g);
-        r[u] = ld_group(ref_row, g);
-      } else if (left > 0) {
-        v[u] = ld_group_ragged(my_row, g, (int)left);
-        r[u] = ld_group_ragged(ref_row, g, (int)left);
+      const int64_t p = p0 + (int64_t)u * kThreads;
+      const int live = live_of(n_params, p, E);
+      if (live > 0) {
+        ld_pack_any(my_row, p, live, v[u]);
+        ld_pack_any(ref_row, p, live, r[u]);
       } else {
-        v[u] = r[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < E; ++i) v[u][i] = r[u][i] = 0.f;
       }
     }
     float a = 0.f, b = 0.f;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const float dx = v[u].x - r[u].x, dy = v[u].y - r[u].y;
-      const float dz = v[u].z - r[u].z, dw = v[u].w - r[u].w;
-      a = fmaf(v[u].x, v[u].x, a); a = fmaf(v[u].y, v[u].y, a);
-      a = fmaf(v[u].z, v[u].z, a); a = fmaf(v[u].w, v[u].w, a);
-      b = fmaf(dx, dx, b); b = fmaf(dy, dy, b);
-      b = fmaf(dz, dz, b); b = fmaf(dw, dw, b);
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        const float d = v[u][i] - r[u][i];
+        a = fmaf(v[u][i], v[u][i], a);
+        b = fmaf(d, d, b);
+      }
     }
     n2 += (double)a;
     d2 += (double)b;
@@ -450,21 +596,150 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
     double s = 0.0;
     for (int wi = 0; wi < kWarps; ++wi) s += s_part[threadIdx.x][wi];
     partials[((int64_t)threadIdx.x * n_devices + row) * lanes + my_lane] = s;
-    __threadfence();
+  }
+  finish_by_last_block(partials, 2 * n_devices, lanes, ticket, &s_last,
+                       [&](int t, double sum) { out[t] = (float)sum; });
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused round: local update of every device, partial aggregation with write-back (optionally
+// sent to every device: global synchronisation) and the statistics, in ONE pass over the arena.
+// Selection only needs the versions, which the host knows before the steps run, so the selected
+// set is an input.  Per pack a thread visits the rows in the order "selected devices in draw
+// order, then the others": it runs each row's steps in registers exactly as K1 does, folds the
+// selected rows into the aggregate in draw order exactly as K2 does (acc = a_0 w_0, then fma),
+// writes the aggregate to the selected rows when the last of them is done, and for every row adds
+// the squares of what the row now holds, and of its distance to the aggregate, to the row's sums.
+// Parameters and momentum come out bit-identical to K1 followed by K2 (and the broadcast); the
+// aggregate is never re-read from memory, so a round moves 16 bytes per (device, parameter)
+// instead of 20 + 8k/N.
+// Grid: persistent, grid-stride over packs.  Row sums: five-shuffle pair reduction per row and
+// pack, accumulated in fp64 in a shared-memory slot owned by the warp; fixed-order sum over warps
+// -> partials[value][block]; last-ticket block finishes.  Deterministic.
+// ------------------------------------------------------------------------------------------
+struct RoundArgs {
+  int32_t n;          // rows visited = all N devices: [0, k) selected in draw order, then the rest
+  int32_t k;          // number of selected devices, 1 <= k <= n
+  int32_t write_all;  // 1: every device receives the aggregate (global synchronisation)
+  float a[kMaxDevices];  // aggregation weights of the selected devices
+  RowStep r[kMaxDevices];
+};
+
+template <typename WT, typename Gen, int E>
+__global__ void __launch_bounds__(kThreads)
+k_round(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_params, RoundArgs a,
+        PhiloxKeys keys, float lr, float mu, float wd, float gstd,
+        double *__restrict__ partials, unsigned int *__restrict__ ticket, float *__restrict__ out) {
+  constexpr int kWarps = kThreads / 32;
+  __shared__ double s_sum[kWarps][2 * kMaxDevices];  // [warp][2 * visit index + which]
+  __shared__ bool s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int t = lane; t < 2 * kMaxDevices; t += 32) s_sum[warp][t] = 0.0;
+  __syncwarp();
+
+  StepConsts k;
+  k.scale2 = gstd * gstd;
+  k.lg_scale = kMinusTwoLn2 * k.scale2;
+  k.neg_lr = -lr;
+  k.mu = mu;
+  k.wd = wd;
+  const int64_t n_packs = (n_params + E - 1) / E;
+  // whole warps iterate together (the shuffles need every lane): round the pack count up to a
+  // multiple of 32; lanes beyond the end carry live = 0 and contribute zeros.
+  const int64_t n_packs_padded = (n_packs + 31) / 32 * 32;
+
+  for (int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x; p < n_packs_padded;
+       p += (int64_t)gridDim.x * kThreads) {
+    const int live = live_of(n_params, p, E);
+    const GroupProducts<E / 4> gp(p);
+    float wv[E], mv[E], wn[E], mn[E], acc[E];
+#pragma unroll
+    for (int i = 0; i < E; ++i) wv[i] = mv[i] = wn[i] = mn[i] = acc[i] = 0.f;
+    if (live > 0) {
+      ld_pack_any(w + (int64_t)a.r[0].row * stride, p, live, wv);
+      if (a.r[0].steps > 0) ld_pack_any(m + (int64_t)a.r[0].row * stride, p, live, mv);
+    }
+    for (int j = 0; j < a.n; ++j) {
+      if (live > 0 && j + 1 < a.n) {
+        ld_pack_any(w + (int64_t)a.r[j + 1].row * stride, p, live, wn);
+        if (a.r[j + 1].steps > 0) ld_pack_any(m + (int64_t)a.r[j + 1].row * stride, p, live, mn);
+      }
+      const bool stepped = a.r[j].steps > 0;
+      if (live > 0 && stepped) {
+        sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+        st_pack_any(m + (int64_t)a.r[j].row * stride, p, live, mv);
+#pragma unroll
+        for (int i = 0; i < E; ++i) wv[i] = i < live ? as_stored(wv[i], w) : 0.f;  // dead lanes stay 0
+      }
+      float n2 = 0.f, d2 = 0.f;
+      bool have_sums = false;
+      if (j < a.k) {
+        const float aj = a.a[j];
+        if (j == 0) {
+#pragma unroll
+          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(aj, wv[i]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
+        }
+        if (j == a.k - 1) {
+          if (a.k > 1 || sizeof(WT) == 2) {
+#pragma unroll
+            for (int i = 0; i < E; ++i) acc[i] = as_stored(acc[i], w);
+          }
+          if (live > 0)
+            for (int t = 0; t < a.k; ++t)
+              if (a.k > 1 || a.r[t].steps > 0)
+                st_pack_any(w + (int64_t)a.r[t].row * stride, p, live, acc);
+#pragma unroll
+          for (int i = 0; i < E; ++i) n2 = fmaf(acc[i], acc[i], n2);
+          have_sums = true;  // one value for all selected rows, stored at visit index k - 1
+        }
+      } else {
+        if (a.write_all) {
+          if (live > 0) st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, acc);
+#pragma unroll
+          for (int i = 0; i < E; ++i) n2 = fmaf(acc[i], acc[i], n2);
+        } else {
+          if (live > 0 && stepped) st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, wv);
+#pragma unroll
+          for (int i = 0; i < E; ++i) {
+            const float d = wv[i] - acc[i];
+            n2 = fmaf(wv[i], wv[i], n2);
+            d2 = fmaf(d, d, d2);
+          }
+        }
+        have_sums = true;
+      }
+      if (have_sums) {
+        const float s = warp_sum_pair(n2, d2, lane);
+        if ((lane & 15) == 0) s_sum[warp][2 * j + (lane >> 4)] += (double)s;
+      }
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        wv[i] = wn[i];
+        mv[i] = mn[i];
+      }
+    }
   }
   __syncthreads();
-  if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  for (int t = warp; t < 2 * n_devices; t += kWarps) {  // t = which * N + row
-    const double *src = partials + (int64_t)t * lanes;
+  // partials[value][block]; value = 2 * visit index + which
+  const int n_vals = 2 * a.n;
+  if ((int)threadIdx.x < n_vals) {
     double s = 0.0;
-    for (int l = lane; l < lanes; l += 32) s += __ldcg(src + l);
-    s = warp_sum(s);
-    if (lane == 0) out[t] = (float)s;
+    for (int wi = 0; wi < kWarps; ++wi) s += s_sum[wi][threadIdx.x];
+    partials[(int64_t)threadIdx.x * gridDim.x + blockIdx.x] = s;
   }
-  if (threadIdx.x == 0) *ticket = 0u;
+  const int n_dev = a.n, ksel = a.k;
+  finish_by_last_block(partials, n_vals, (int)gridDim.x, ticket, &s_last, [&](int t, double sum) {
+    const int j = t >> 1, which = t & 1;
+    if (j < ksel - 1) return;  // selected rows share the value kept at visit index k - 1
+    if (j == ksel - 1) {
+      for (int q = 0; q < ksel; ++q) out[which * n_dev + a.r[q].row] = which ? 0.f : (float)sum;
+    } else {
+      out[which * n_dev + a.r[j].row] = (float)sum;
+    }
+  });
 }
 
 // ------------------------------------------------------------------------------------------

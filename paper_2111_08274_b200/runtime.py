@@ -41,10 +41,17 @@ class Arena:
             self.h.destroy()
             self.h = None
 
+    def run_round_fused(self, r):
+        """The same round as run_round through the single fused kernel (hadfl_round)."""
+        wl = self.wl
+        sync = bool(wl.sync_every) and (r + 1) % wl.sync_every == 0
+        return self.h.round(self.ids, wl.steps_for_round(r), wl.lr, r, wl.k, self.select_seed,
+                            sync_all=sync)
+
     def run_round(self, r, stats=True):
-        """One round of the hot path: local steps of every device, selection, aggregation with
-        write-back (plus, on the workload's global-synchronisation rounds, the send to the
-        unselected devices), statistics.  Returns the selected ids (draw order)."""
+        """One round of the hot path as separate calls: local steps of every device, selection,
+        aggregation with write-back (plus, on the workload's global-synchronisation rounds, the
+        send to the unselected devices), statistics.  Returns the selected ids (draw order)."""
         wl, h = self.wl, self.h
         h.local_step(self.ids, wl.steps_for_round(r), wl.lr)
         sel = h.select(r, wl.k, self.select_seed)

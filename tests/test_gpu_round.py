@@ -1,0 +1,129 @@
+"""The fused round kernel (hadfl_round) against the separate calls it replaces and against the CPU
+oracle: selections, versions, parameters and momentum must equal the unfused sequence bit for bit;
+its statistics agree with the oracle's double-precision sums to 1e-5."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_common import assert_close_params, bf16_ulp, require_gpu
+from oracle_driver import make_sim, oracle_round
+from paper_2111_08274_b200 import binding, runtime, workloads
+from paper_2111_08274_b200.workloads import Workload
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def wl_of(n, P, k, dtype=0, steps=None, sync_every=0, **kw):
+    steps = tuple(1 + (3 * i) % 5 for i in range(n)) if steps is None else steps
+    return Workload("rt", n, P, k, 6, "fixed", steps, grad_std=1e-2, dtype=dtype,
+                    seed=workloads.BASE_SEED + 31 * n + P, sync_every=sync_every, **kw)
+
+
+def assert_same_state(a, b, n):
+    for i in range(n):
+        assert np.array_equal(a.h.read_params(i), b.h.read_params(i)), i
+        assert np.array_equal(a.h.read_momentum(i), b.h.read_momentum(i)), i
+    va, vb = a.h.get_versions(), b.h.get_versions()
+    assert np.array_equal(va[0], vb[0]) and np.array_equal(va[1], vb[1])
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("n,P,k", [(4, 100_003, 2), (8, 70_001, 4), (16, 33_333, 1), (32, 9_999, 16),
+                                   (32, 4_099, 32), (1, 5, 1), (5, 1, 3), (6, 300_007, 3)])
+def test_fused_round_equals_separate_calls(oracle, n, P, k, dtype):
+    wl = wl_of(n, P, k, dtype=dtype, sync_every=3)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    sim = make_sim(oracle, wl)
+    for r in range(wl.rounds):
+        sf = fused.run_round_fused(r)
+        sp = plain.run_round(r)
+        so = oracle_round(sim, wl, r)
+        assert np.array_equal(sf, sp) and np.array_equal(sf, so), r
+        n2, d2 = fused.h.stats_read()
+        pn2, pd2 = plain.h.stats_read()
+        on2, od2 = sim.stats(int(so[0]))
+        assert np.allclose(n2, pn2, rtol=2e-6) and np.allclose(d2, pd2, rtol=2e-6, atol=1e-30), r
+        if dtype == 0:
+            assert np.allclose(n2, on2, rtol=1e-5) and np.allclose(d2, od2, rtol=1e-5, atol=1e-12), r
+        assert all(d2[int(s)] == 0.0 for s in sf)
+    assert_same_state(fused, plain, n)
+    if dtype == 0:
+        for i in range(n):
+            assert_close_params(fused.h.read_params(i), sim.read_params(i), "w[%d]" % i)
+    else:
+        for i in range(n):
+            got, want = fused.h.read_params(i), sim.read_params(i)
+            assert np.abs(got - want).max() <= 2 * bf16_ulp(np.abs(want).max()) and np.mean(got != want) < 0.02
+    fused.close()
+    plain.close()
+
+
+def test_fused_round_subset_of_devices_zero_steps_mask_and_versions(oracle):
+    """Only some devices step, one of them zero steps; an availability mask; caller-supplied versions."""
+    wl = wl_of(6, 20_003, 2)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    mask = [1, 1, 0, 1, 1, 1]
+    for ar in (fused, plain):
+        ar.h.set_available(mask)
+    ids, steps = [4, 0, 2], [3, 0, 2]
+    pv = [2.0, 2.5, 9.0, 1.0, 3.0, 3.0]
+    for r, versions in ((0, None), (1, pv), (2, None)):
+        sf = fused.h.round(ids, steps, 0.01, r, 2, 77, versions=versions)
+        plain.h.local_step(ids, steps, 0.01)
+        sp = plain.h.select(r, 2, 77, versions)
+        plain.h.aggregate(sp, versions)
+        plain.h.stats_enqueue(int(sp[0]))
+        assert np.array_equal(sf, sp) and 2 not in sf
+        a, b = fused.h.stats_read(), plain.h.stats_read()
+        assert np.allclose(a[0], b[0], rtol=2e-6) and np.allclose(a[1], b[1], rtol=2e-6, atol=1e-30)
+    assert_same_state(fused, plain, 6)
+    fused.close()
+    plain.close()
+
+
+def test_fused_round_version_weighted_mode():
+    wl = wl_of(8, 12_345, 4, weight_mode=1, version_scale=0.5)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    for r in range(4):
+        assert np.array_equal(fused.run_round_fused(r), plain.run_round(r))
+    assert_same_state(fused, plain, 8)
+    fused.close()
+    plain.close()
+
+
+def test_fused_round_is_reproducible_and_rejects_bad_arguments():
+    wl = wl_of(8, 50_001, 4)
+    a, b = runtime.Arena(wl), runtime.Arena(wl)
+    for r in range(3):
+        a.run_round_fused(r)
+        b.run_round_fused(r)
+        sa, sb = a.h.stats_read(), b.h.stats_read()
+        assert np.array_equal(sa[0], sb[0]) and np.array_equal(sa[1], sb[1])     # bit for bit
+    assert_same_state(a, b, 8)
+    before = a.h.read_params(3)
+    E = binding.HadflError
+    for ids, steps, k in (([0, 0], [1, 1], 2), ([8], [1], 2), ([0], [-1], 2), ([0], [1], 0), ([0], [1], 9), ([], [], 2)):
+        with pytest.raises(E):
+            a.h.round(ids, steps, 0.01, 5, k, 1)
+    assert np.array_equal(a.h.read_params(3), before)
+    a.close()
+    b.close()
+
+
+def test_fused_round_counter_crossing_falls_back_to_separate_kernels():
+    wl = wl_of(3, 4_099, 2)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    start = np.array([2**32 - 2, 5, 2**33 - 1], dtype=np.uint64)
+    for ar in (fused, plain):
+        ar.h.set_versions(step_counts=start)
+    sf = fused.run_round_fused(0)
+    sp = plain.run_round(0)
+    assert np.array_equal(sf, sp)
+    assert_same_state(fused, plain, 3)
+    fused.close()
+    plain.close()
