@@ -44,19 +44,34 @@ struct hadfl_handle {
 
 namespace {
 
+inline size_t elem_size(const hadfl_handle *h) { return h->cfg.dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
+
 constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
 
-// Columns per thread in the local-update and fused-round kernels: one Philox block for fp32
-// storage, two (one 16-byte access of w) for bf16 storage.
+// Columns per thread in the local-update and fused-round kernels: two Philox blocks (two 16-byte
+// accesses of fp32 w, one of bf16 w).  Two independent generator chains per thread give the
+// scheduler more to issue, and the per-row overhead is spread over twice the elements.
 template <typename WT>
 struct StepPack {
-  static constexpr int E = Pack16<WT>::E;
+  static constexpr int E = 8;
 };
+
+StepConsts step_consts(const hadfl_handle *h, float lr) {
+  StepConsts k;
+  k.neg_lr = -lr;
+  k.mu = h->cfg.momentum;
+  k.wd = h->cfg.weight_decay;
+  k.scale2 = h->cfg.grad_std * h->cfg.grad_std;
+  k.lg_scale = kMinusTwoLn2 * k.scale2;
+  return k;
+}
 
 // What the kernels need to know about one device's steps in one launch.
 RowStep row_step(const hadfl_handle *h, int dev, uint64_t base, int steps) {
   const uint64_t dp = (uint64_t)kPhiloxM1 * (uint32_t)dev;
   RowStep r;
+  r.w_off = (int64_t)dev * h->stride * (int64_t)elem_size(h);
+  r.m_off = (int64_t)dev * h->stride * (int64_t)sizeof(float);
   r.row = dev;
   r.steps = steps;
   r.base_lo = (uint32_t)base;
@@ -86,8 +101,6 @@ struct DeviceGuard {
     if (switched) cudaSetDevice(prev);
   }
 };
-
-inline size_t elem_size(const hadfl_handle *h) { return h->cfg.dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
 
 bool distinct_ids(const hadfl_handle *h, const int32_t *ids, int n) {
   if (!ids || n < 1 || n > h->cfg.n_devices) return false;
@@ -126,24 +139,25 @@ int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
   const int64_t packs = (h->cfg.n_params + E - 1) / E;
   const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
   k_local_step<WT, NormalsFast, E><<<blocks, kThreads, 0, h->stream>>>(
-      (WT *)h->w, h->m, h->stride, h->cfg.n_params, a, h->keys, lr, h->cfg.momentum,
-      h->cfg.weight_decay, h->cfg.grad_std);
+      (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
   return check_launch(h);
 }
 
 template <typename WT>
 int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
-  k_round<WT, NormalsFast, StepPack<WT>::E><<<h->round_grid, kThreads, 0, h->stream>>>(
-      (WT *)h->w, h->m, h->stride, h->cfg.n_params, a, h->keys, lr, h->cfg.momentum,
-      h->cfg.weight_decay, h->cfg.grad_std, h->d_round_partials, h->d_round_ticket, h->d_stats);
+  const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
+  k_round<WT, NormalsFast, StepPack<WT>::E><<<h->round_grid, kThreads, smem, h->stream>>>(
+      (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+      h->d_round_ticket, h->d_stats);
   return check_launch(h);
 }
 
 template <typename WT>
-int round_blocks_per_sm() {
+int round_blocks_per_sm(int n_devices) {
   int n = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-          &n, k_round<WT, NormalsFast, StepPack<WT>::E>, kThreads, 0) != cudaSuccess || n < 1)
+          &n, k_round<WT, NormalsFast, StepPack<WT>::E>, kThreads,
+          sizeof(float) * kThreads * (size_t)n_devices) != cudaSuccess || n < 1)
     n = 1;
   return n;
 }
@@ -294,8 +308,9 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
   // Fused round kernel: one resident wave, never more blocks than there are packs to visit.
   {
-    const int per_sm = cfg->dtype == HADFL_DTYPE_BF16 ? round_blocks_per_sm<__nv_bfloat16>()
-                                                      : round_blocks_per_sm<float>();
+    const int per_sm = cfg->dtype == HADFL_DTYPE_BF16
+                           ? round_blocks_per_sm<__nv_bfloat16>(cfg->n_devices)
+                           : round_blocks_per_sm<float>(cfg->n_devices);
     int64_t grid = (int64_t)h->sm_count * per_sm;
     const int64_t need = (packs + kThreads - 1) / kThreads;
     if (grid > need) grid = need;

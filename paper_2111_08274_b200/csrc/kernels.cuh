@@ -317,6 +317,8 @@ k_init(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_para
 // cross a multiple of 2^32 inside one launch (it splits the call), so the step index is one add.
 // ------------------------------------------------------------------------------------------
 struct RowStep {
+  int64_t w_off;     // byte offset of the device's row in the parameter arena
+  int64_t m_off;     // byte offset of the device's row in the momentum arena
   int32_t row;
   int32_t steps;
   uint32_t base_lo;  // low word of the device's step counter before this call
@@ -330,6 +332,8 @@ struct LocalStepArgs {
   RowStep r[kMaxDevices];
 };
 
+// Constants of the update, computed once on the host and read from the launch parameters:
+// -lr, momentum, weight decay, -2 ln2 grad_std^2 and grad_std^2.
 struct StepConsts {
   float neg_lr, mu, wd, lg_scale, scale2;
 };
@@ -375,40 +379,46 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
   }
 }
 
+// Row addressing: the host passes each row's byte offset, the thread adds the byte offset of its
+// pack once, so a row access costs one 64-bit add.  The row loop is unrolled by two with the two
+// register sets (current row / prefetched row) swapping roles, so nothing is copied.
+template <typename WT>
+__device__ __forceinline__ WT *at_row(char *pack_in_row0, int64_t row_off) {
+  return reinterpret_cast<WT *>(pack_in_row0 + row_off);
+}
+
 template <typename WT, typename Gen, int E>
 __global__ void __launch_bounds__(kThreads)
-k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_params,
-             LocalStepArgs a, PhiloxKeys keys, float lr, float mu, float wd, float gstd) {
+k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalStepArgs a,
+             PhiloxKeys keys, StepConsts k) {
   const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   const int live = live_of(n_params, p, E);
   if (live == 0) return;
   const GroupProducts<E / 4> gp(p);
-  StepConsts k;
-  k.scale2 = gstd * gstd;
-  k.lg_scale = kMinusTwoLn2 * k.scale2;
-  k.neg_lr = -lr;
-  k.mu = mu;
-  k.wd = wd;
+  char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
+  char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(float));
 
-  float wv[E], mv[E], wn[E], mn[E];
-  ld_pack_any(w + (int64_t)a.r[0].row * stride, p, live, wv);
-  ld_pack_any(m + (int64_t)a.r[0].row * stride, p, live, mv);
-  for (int j = 0; j < a.n; ++j) {
-    if (j + 1 < a.n) {
-      ld_pack_any(w + (int64_t)a.r[j + 1].row * stride, p, live, wn);
-      ld_pack_any(m + (int64_t)a.r[j + 1].row * stride, p, live, mn);
-    }
+  auto load = [&](int j, float (&wv)[E], float (&mv)[E]) {
+    ld_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+    ld_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+  };
+  auto visit = [&](int j, float (&wv)[E], float (&mv)[E]) {
     if (a.r[j].steps > 0) {
       sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-      st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, wv);
-      st_pack_any(m + (int64_t)a.r[j].row * stride, p, live, mv);
+      st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+      st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
     }
-#pragma unroll
-    for (int i = 0; i < E; ++i) {
-      wv[i] = wn[i];
-      mv[i] = mn[i];
-    }
+  };
+  float w0[E], m0[E], w1[E], m1[E];
+  load(0, w0, m0);
+  int j = 0;
+  for (; j + 1 < a.n; j += 2) {
+    load(j + 1, w1, m1);
+    visit(j, w0, m0);
+    if (j + 2 < a.n) load(j + 2, w0, m0);
+    visit(j + 1, w1, m1);
   }
+  if (j < a.n) visit(j, w0, m0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -613,9 +623,10 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 // Parameters and momentum come out bit-identical to K1 followed by K2 (and the broadcast); the
 // aggregate is never re-read from memory, so a round moves 16 bytes per (device, parameter)
 // instead of 20 + 8k/N.
-// Grid: persistent, grid-stride over packs.  Row sums: five-shuffle pair reduction per row and
-// pack, accumulated in fp64 in a shared-memory slot owned by the warp; fixed-order sum over warps
-// -> partials[value][block]; last-ticket block finishes.  Deterministic.
+// Grid: persistent, grid-stride over packs.  Row sums: one shuffle per row and pack, then a
+// shared-memory slot owned by the thread (fp32); at the end a butterfly over each half-warp, a
+// fixed-order fp64 sum over warps -> partials[value][block]; last-ticket block finishes.
+// Deterministic.  Dynamic shared memory: n * kThreads floats.
 // ------------------------------------------------------------------------------------------
 struct RoundArgs {
   int32_t n;          // rows visited = all N devices: [0, k) selected in draw order, then the rest
@@ -625,55 +636,62 @@ struct RoundArgs {
   RowStep r[kMaxDevices];
 };
 
+// Adds a thread's (sum of squares, sum of squared distances) for one row to the block's
+// accumulators.  One shuffle folds lane l and lane l ^ 16 so that the lower half-warp carries the
+// first value and the upper half the second; each thread then owns ONE fp32 slot per row,
+// s_acc[visit index][thread], which it alone updates (no atomics, fixed order).
+__device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, float d2, int lane) {
+  const bool upper = (lane & 16) != 0;
+  const float keep = upper ? d2 : n2;
+  const float give = upper ? n2 : d2;
+  float *slot = s_acc + j * kThreads + threadIdx.x;
+  *slot += keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
+}
+
 template <typename WT, typename Gen, int E>
 __global__ void __launch_bounds__(kThreads)
-k_round(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_params, RoundArgs a,
-        PhiloxKeys keys, float lr, float mu, float wd, float gstd,
-        double *__restrict__ partials, unsigned int *__restrict__ ticket, float *__restrict__ out) {
+k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
+        StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
+        float *__restrict__ out) {
   constexpr int kWarps = kThreads / 32;
+  extern __shared__ float s_acc[];                   // [a.n][kThreads]: per-thread row sums
   __shared__ double s_sum[kWarps][2 * kMaxDevices];  // [warp][2 * visit index + which]
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int t = lane; t < 2 * kMaxDevices; t += 32) s_sum[warp][t] = 0.0;
-  __syncwarp();
+  for (int j = 0; j < a.n; ++j) s_acc[j * kThreads + threadIdx.x] = 0.f;
 
-  StepConsts k;
-  k.scale2 = gstd * gstd;
-  k.lg_scale = kMinusTwoLn2 * k.scale2;
-  k.neg_lr = -lr;
-  k.mu = mu;
-  k.wd = wd;
   const int64_t n_packs = (n_params + E - 1) / E;
-  // whole warps iterate together (the shuffles need every lane): round the pack count up to a
-  // multiple of 32; lanes beyond the end carry live = 0 and contribute zeros.
+  // Whole warps iterate together (the row sums use a shuffle): the pack count is rounded up to a
+  // multiple of 32; lanes beyond the end carry live = 0, load and store nothing, and add zeros.
   const int64_t n_packs_padded = (n_packs + 31) / 32 * 32;
 
   for (int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x; p < n_packs_padded;
        p += (int64_t)gridDim.x * kThreads) {
     const int live = live_of(n_params, p, E);
+    const bool act = live > 0;
     const GroupProducts<E / 4> gp(p);
-    float wv[E], mv[E], wn[E], mn[E], acc[E];
+    char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
+    char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(float));
+    float acc[E];
 #pragma unroll
-    for (int i = 0; i < E; ++i) wv[i] = mv[i] = wn[i] = mn[i] = acc[i] = 0.f;
-    if (live > 0) {
-      ld_pack_any(w + (int64_t)a.r[0].row * stride, p, live, wv);
-      if (a.r[0].steps > 0) ld_pack_any(m + (int64_t)a.r[0].row * stride, p, live, mv);
-    }
-    for (int j = 0; j < a.n; ++j) {
-      if (live > 0 && j + 1 < a.n) {
-        ld_pack_any(w + (int64_t)a.r[j + 1].row * stride, p, live, wn);
-        if (a.r[j + 1].steps > 0) ld_pack_any(m + (int64_t)a.r[j + 1].row * stride, p, live, mn);
+    for (int i = 0; i < E; ++i) acc[i] = 0.f;
+
+    auto load = [&](int j, float (&wv)[E], float (&mv)[E]) {
+      if (act) {
+        ld_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+        if (a.r[j].steps > 0) ld_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
       }
-      const bool stepped = a.r[j].steps > 0;
-      if (live > 0 && stepped) {
+    };
+    // One row: its steps, then its part in the aggregation / synchronisation and in the sums.
+    auto visit = [&](int j, float (&wv)[E], float (&mv)[E]) {
+      const bool stepped = act && a.r[j].steps > 0;
+      if (stepped) {
         sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-        st_pack_any(m + (int64_t)a.r[j].row * stride, p, live, mv);
+        st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
 #pragma unroll
         for (int i = 0; i < E; ++i) wv[i] = i < live ? as_stored(wv[i], w) : 0.f;  // dead lanes stay 0
       }
-      float n2 = 0.f, d2 = 0.f;
-      bool have_sums = false;
-      if (j < a.k) {
+      if (j < a.k) {  // a selected device, visited in draw order: fold into the aggregate
         const float aj = a.a[j];
         if (j == 0) {
 #pragma unroll
@@ -683,58 +701,66 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_par
           for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
         }
         if (j == a.k - 1) {
-          if (a.k > 1 || sizeof(WT) == 2) {
-#pragma unroll
-            for (int i = 0; i < E; ++i) acc[i] = as_stored(acc[i], w);
-          }
-          if (live > 0)
-            for (int t = 0; t < a.k; ++t)
-              if (a.k > 1 || a.r[t].steps > 0)
-                st_pack_any(w + (int64_t)a.r[t].row * stride, p, live, acc);
-#pragma unroll
-          for (int i = 0; i < E; ++i) n2 = fmaf(acc[i], acc[i], n2);
-          have_sums = true;  // one value for all selected rows, stored at visit index k - 1
-        }
-      } else {
-        if (a.write_all) {
-          if (live > 0) st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, acc);
-#pragma unroll
-          for (int i = 0; i < E; ++i) n2 = fmaf(acc[i], acc[i], n2);
-        } else {
-          if (live > 0 && stepped) st_pack_any(w + (int64_t)a.r[j].row * stride, p, live, wv);
+          float n2 = 0.f;
 #pragma unroll
           for (int i = 0; i < E; ++i) {
-            const float d = wv[i] - acc[i];
-            n2 = fmaf(wv[i], wv[i], n2);
-            d2 = fmaf(d, d, d2);
+            acc[i] = as_stored(acc[i], w);
+            n2 = fmaf(acc[i], acc[i], n2);
           }
+          // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
+          if (act && (a.k > 1 || a.r[0].steps > 0))
+            for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
+          add_row_sums(s_acc, j, n2, 0.f, lane);  // one value for all selected devices
         }
-        have_sums = true;
-      }
-      if (have_sums) {
-        const float s = warp_sum_pair(n2, d2, lane);
-        if ((lane & 15) == 0) s_sum[warp][2 * j + (lane >> 4)] += (double)s;
-      }
+      } else {  // another device: keep its own model, or receive the aggregate
+        if (a.write_all) {
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        wv[i] = wn[i];
-        mv[i] = mn[i];
+          for (int i = 0; i < E; ++i) wv[i] = acc[i];
+        }
+        if (act && (stepped || a.write_all)) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+        float n2 = 0.f, d2 = 0.f;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+          const float d = wv[i] - acc[i];
+          n2 = fmaf(wv[i], wv[i], n2);
+          d2 = fmaf(d, d, d2);
+        }
+        add_row_sums(s_acc, j, n2, d2, lane);
       }
+    };
+    float w0[E], m0[E], w1[E], m1[E];
+#pragma unroll
+    for (int i = 0; i < E; ++i) w0[i] = m0[i] = w1[i] = m1[i] = 0.f;
+    load(0, w0, m0);
+    int j = 0;
+    for (; j + 1 < a.n; j += 2) {
+      load(j + 1, w1, m1);
+      visit(j, w0, m0);
+      if (j + 2 < a.n) load(j + 2, w0, m0);
+      visit(j + 1, w1, m1);
     }
+    if (j < a.n) visit(j, w0, m0);
+  }
+  // ---- block: fold the per-thread slots (lower half-warps hold norms, upper halves distances)
+  for (int j = a.k - 1; j < a.n; ++j) {
+    float v = s_acc[j * kThreads + threadIdx.x];
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    if ((lane & 15) == 0) s_sum[warp][2 * j + (lane >> 4)] = (double)v;
   }
   __syncthreads();
   // partials[value][block]; value = 2 * visit index + which
   const int n_vals = 2 * a.n;
-  if ((int)threadIdx.x < n_vals) {
+  if ((int)threadIdx.x < n_vals && (int)threadIdx.x >= 2 * (a.k - 1)) {
     double s = 0.0;
     for (int wi = 0; wi < kWarps; ++wi) s += s_sum[wi][threadIdx.x];
     partials[(int64_t)threadIdx.x * gridDim.x + blockIdx.x] = s;
   }
   const int n_dev = a.n, ksel = a.k;
-  finish_by_last_block(partials, n_vals, (int)gridDim.x, ticket, &s_last, [&](int t, double sum) {
-    const int j = t >> 1, which = t & 1;
-    if (j < ksel - 1) return;  // selected rows share the value kept at visit index k - 1
-    if (j == ksel - 1) {
+  finish_by_last_block(partials + (int64_t)2 * (ksel - 1) * gridDim.x, n_vals - 2 * (ksel - 1),
+                       (int)gridDim.x, ticket, &s_last, [&](int t, double sum) {
+    const int j = ksel - 1 + (t >> 1), which = t & 1;
+    if (j == ksel - 1) {  // the selected devices share one norm and are at distance 0
       for (int q = 0; q < ksel; ++q) out[which * n_dev + a.r[q].row] = which ? 0.f : (float)sum;
     } else {
       out[which * n_dev + a.r[j].row] = (float)sum;

@@ -6,7 +6,8 @@
 The arena (N * P * 8 bytes for fp32) should exceed the 126 MB L2 so that DRAM counters mean
 something, and stay at a few hundred MB so that a multi-pass capture ends quickly.
 Launch order per repetition: local update once per entry of --steps (all devices that many
-steps), aggregation of k devices, statistics, broadcast to the other devices.
+steps), aggregation of k devices, statistics, broadcast to the other devices.  With --fused: one
+hadfl_round launch per entry of --steps instead.
 """
 import argparse
 
@@ -23,6 +24,7 @@ def main():
     ap.add_argument("--steps", type=str, default="1,8")
     ap.add_argument("--dtype", type=int, default=0)
     ap.add_argument("--reps", type=int, default=2)
+    ap.add_argument("--fused", action="store_true", help="run hadfl_round instead of the separate calls")
     a = ap.parse_args()
     wl = workloads.Workload("profile", a.n, a.p, a.k, 1, "fixed", (1,) * a.n, dtype=a.dtype,
                             seed=workloads.BASE_SEED)
@@ -30,7 +32,10 @@ def main():
     ar = runtime.Arena(wl)
     ids = wl.device_ids()
     sel = ids[: a.k]
-    for _ in range(a.reps):
+    for rep in range(a.reps if a.fused else 0):
+        for s in [int(t) for t in a.steps.split(",")]:
+            ar.h.round(ids, np.full(a.n, s, dtype=np.int32), wl.lr, rep, a.k, 1)
+    for _ in range(0 if a.fused else a.reps):
         for s in [int(t) for t in a.steps.split(",")]:
             ar.h.local_step(ids, np.full(a.n, s, dtype=np.int32), wl.lr)
         ar.h.aggregate(sel)

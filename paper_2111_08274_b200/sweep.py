@@ -3,8 +3,9 @@
     python -m paper_2111_08274_b200.sweep [--what c5|configs|all] [--rounds 30] [--json out.json]
 
 For every case: warm-up rounds, then `--rounds` timed rounds with CUDA events around each launch.
-Prints markdown tables: per kernel the average launch time and the algorithmic GB/s (bytes that
-must move / time), and the rounds/s of the whole round.  Small vectors (arena below the 126 MB L2)
+Prints markdown tables: per kernel the median launch time and the algorithmic GB/s (bytes that
+must move / time), the rounds/s of the round as separate calls, and the rounds/s of the same
+round through the fused kernel (its GB/s counts 16 bytes per device and parameter).  Small vectors (arena below the 126 MB L2)
 are L2- and launch-bound and are reported as such, not as HBM bandwidth.
 """
 import argparse
@@ -44,11 +45,25 @@ def measure(wl, rounds, warmup=3):
     torch.cuda.synchronize()
     ms = {n: float(np.median([a.elapsed_time(b) for a, b in ev[n]])) for n in names}
     total_ms = start.elapsed_time(end) / rounds
+    r += rounds
+    # the same rounds through the fused kernel
+    for i in range(warmup):
+        arena.run_round_fused(r + i)
+    r += warmup
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(rounds):
+        arena.run_round_fused(r + i)
+    end.record()
+    torch.cuda.synchronize()
+    fused_ms = start.elapsed_time(end) / rounds
     bytes_ = {"local_step": N * P * (2 * ew + 8), "aggregate": 2 * k * P * ew, "stats": N * P * ew}
     arena.close()
     res = {"workload": wl.name, "N": N, "P": P, "k": k, "storage": "bf16" if wl.dtype else "fp32",
            "mean_steps": float(np.mean([s.mean() for s in steps])),
-           "arena_mb": N * P * (ew + 4) / 1e6, "round_ms": total_ms, "rounds_per_s": 1e3 / total_ms}
+           "arena_mb": N * P * (ew + 4) / 1e6, "round_ms": total_ms, "rounds_per_s": 1e3 / total_ms,
+           "fused_round_ms": fused_ms, "fused_rounds_per_s": 1e3 / fused_ms,
+           "fused_gbs": N * P * (2 * ew + 8) / fused_ms / 1e6}
     for n in names:
         res[n + "_us"] = ms[n] * 1e3
         res[n + "_gbs"] = bytes_[n] / ms[n] / 1e6
@@ -56,15 +71,16 @@ def measure(wl, rounds, warmup=3):
 
 
 def table(rows, peak):
-    out = ["| workload | N | P | k | storage | mean steps | arena MB | K1 µs | K1 GB/s (%% of %.0f) | K2 µs | K2 GB/s (%%) | K3 µs | K3 GB/s (%%) | round ms | rounds/s |" % peak,
-           "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+    out = ["| workload | N | P | k | storage | mean steps | arena MB | K1 µs | K1 GB/s (%% of %.0f) | K2 µs | K2 GB/s (%%) | K3 µs | K3 GB/s (%%) | round ms | rounds/s | fused round ms | fused rounds/s | fused GB/s (%%) |" % peak,
+           "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
     for r in rows:
-        out.append("| %s | %d | %d | %d | %s | %.2f | %.0f | %.1f | %.0f (%.0f) | %.1f | %.0f (%.0f) | %.1f | %.0f (%.0f) | %.3f | %.0f |" % (
+        out.append("| %s | %d | %d | %d | %s | %.2f | %.0f | %.1f | %.0f (%.0f) | %.1f | %.0f (%.0f) | %.1f | %.0f (%.0f) | %.3f | %.0f | %.3f | %.0f | %.0f (%.0f) |" % (
             r["workload"], r["N"], r["P"], r["k"], r["storage"], r["mean_steps"], r["arena_mb"],
             r["local_step_us"], r["local_step_gbs"], 100 * r["local_step_gbs"] / peak,
             r["aggregate_us"], r["aggregate_gbs"], 100 * r["aggregate_gbs"] / peak,
             r["stats_us"], r["stats_gbs"], 100 * r["stats_gbs"] / peak,
-            r["round_ms"], r["rounds_per_s"]))
+            r["round_ms"], r["rounds_per_s"], r["fused_round_ms"], r["fused_rounds_per_s"],
+            r["fused_gbs"], 100 * r["fused_gbs"] / peak))
     return "\n".join(out)
 
 
