@@ -3,17 +3,20 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
 
 A "step" is one round of the whole hot path over one synthetic workload: local update of every
-device with its own step count (K1), selection (host), aggregation with write-back (K2), version
-update and per-replica statistics (K3).  Prints ONE JSON line (rank 0).
+device with its own step count, selection (host), aggregation with write-back, version update and
+per-replica statistics - one hadfl_round call, one kernel launch.  Prints ONE JSON line (rank 0).
 
   value     rounds/s with everything resident in HBM; timed with CUDA events on the library's
             stream, barrier + synchronize on both sides, max over ranks.
+  kernels / separate_calls   the same rounds as separate calls (hadfl_local_step, hadfl_select,
+            hadfl_aggregate, hadfl_stats_enqueue) with CUDA events around every launch: the
+            bandwidth of each kernel on its own.
   e2e       the same rounds through the C ABI with HOST buffers: every round also reads the
             statistics (2N floats) and the aggregated model (P floats, the coordinator's model
             backup) into pinned host memory.
-  roofline  for the kernel with the largest share of the timed region: algorithmic bytes per
-            launch / average launch time (CUDA events around each launch), against the measured
-            copy bandwidth of this machine's B200s.
+  roofline  for the kernel of the timed region (the fused round): algorithmic bytes per launch /
+            average launch time (CUDA events around each launch), against the measured copy
+            bandwidth of this machine's B200s.
   cpu_baseline  the CPU checker (single thread, as it stands) on a column sample of the same
             workload, scaled to the full vector.
 
@@ -39,13 +42,19 @@ from paper_2111_08274_b200 import workloads  # noqa: E402
 METRIC = "aggregation_rounds_per_sec"
 UNIT = "rounds/s"
 FALLBACK_HBM_GBS = 6650.0
+# Arithmetic roofline of the local update: instruction issue.  One step of one Philox block
+# (4 parameters) needs at least 82 warp instructions (9 Philox rounds x (2 wide multiplies +
+# 2 three-input xors) = 36, Box-Muller for two pairs = 28, the update = 12, step loop = 6), i.e.
+# 20.5 per parameter and step; an SM issues 4 x 32 = 128 lane-instructions per clock.
+ALU_INSTR_PER_ELEM_STEP = 20.5
+SM_COUNT, LANES_PER_CLK_PER_SM, SM_MAX_GHZ = 148, 128, 1.965
 ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to size its sample
 
 # DRAM bytes per (device, parameter) moved by one launch, from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same kernel;
 # reads grow in proportion to the elements processed; writes are undercounted by whatever is still
 # dirty in the 126 MB L2 when the kernel ends).  None = not captured for the kernel as it stands.
-NCU_DRAM_BYTES_PER_ELEM = {"local_step": 14.31, "aggregate": 4.50, "stats": 4.12}
+NCU_DRAM_BYTES_PER_ELEM = {"round": None, "local_step": None, "aggregate": 4.50, "stats": 4.12}
 
 
 def measured_peak():
@@ -228,59 +237,103 @@ def run_ours(args, wl):
         r += 1
 
     K = args.steps
-    names = ("local_step", "aggregate", "stats")
-    ev = {n: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-              for _ in range(K)] for n in names}
+    ids, seed = arena.ids, arena.select_seed
+    peak, peak_kind = measured_peak()
+    frac_key = "frac_of_%s_hbm" % peak_kind
+
+    # ---- timed region: K rounds, each ONE call of the public API (hadfl_round: local steps of
+    # every device, selection, aggregation with write-back, version update, statistics) ----------
+    ev_round = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in range(K)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(physical_gpu_index(local))
-    ids, seed = arena.ids, arena.select_seed
     step_lists = [wl.steps_for_round(r + i) for i in range(K)]
+    syncs = [bool(wl.sync_every) and (r + i + 1) % wl.sync_every == 0 for i in range(K)]
     barrier()
     launches0 = h.launch_count()
     sampler.start()
     start.record()
     for i in range(K):
-        a, b = ev["local_step"][i]
-        a.record(); h.local_step(ids, step_lists[i], wl.lr); b.record()
-        sel = h.select(r + i, k, seed)
-        a, b = ev["aggregate"][i]
-        a.record(); h.aggregate(sel); b.record()
-        a, b = ev["stats"][i]
-        a.record(); h.stats_enqueue(int(sel[0])); b.record()
+        a, b = ev_round[i]
+        a.record(); h.round(ids, step_lists[i], wl.lr, r + i, k, seed, sync_all=syncs[i]); b.record()
     end.record()
     barrier()
     clocks = sampler.stop()
     launches = h.launch_count() - launches0
     r += K
     elapsed_ms = max_over_ranks(start.elapsed_time(end), world)
-
-    kern_ms = {n: float(np.mean([a.elapsed_time(b) for a, b in ev[n]])) for n in names}
     mean_steps = float(np.mean([s.sum() for s in step_lists])) / N
+    round_ms = float(np.mean([a.elapsed_time(b) for a, b in ev_round]))
+    round_bytes = N * P * (2 * elem_w + 8)             # w and m read and written once per round
+    round_gbs = round_bytes / (round_ms * 1e-3) / 1e9
+
+    # ---- the same rounds as separate calls, to time each kernel on its own ---------------------
+    Ks = max(3, min(K, 200))
+    names = ("local_step", "aggregate", "stats")
+    ev = {n: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(Ks)] for n in names}
+    sstart, send = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sep_steps = [wl.steps_for_round(r + i) for i in range(Ks)]
+    barrier()
+    sstart.record()
+    for i in range(Ks):
+        a, b = ev["local_step"][i]
+        a.record(); h.local_step(ids, sep_steps[i], wl.lr); b.record()
+        sel = h.select(r + i, k, seed)
+        a, b = ev["aggregate"][i]
+        a.record(); h.aggregate(sel); b.record()
+        a, b = ev["stats"][i]
+        a.record(); h.stats_enqueue(int(sel[0])); b.record()
+    send.record()
+    barrier()
+    r += Ks
+    sep_ms = max_over_ranks(sstart.elapsed_time(send), world) / Ks
+    kern_ms = {n: float(np.mean([a.elapsed_time(b) for a, b in ev[n]])) for n in names}
+    sep_mean_steps = float(np.mean([s.sum() for s in sep_steps])) / N
     alg_bytes = {"local_step": N * P * (2 * elem_w + 8),       # read + write w and m, once per call
                  "aggregate": 2 * k * P * elem_w,              # k rows read, k rows written
                  "stats": N * P * elem_w}                      # every row read once
     units = {"local_step": N * P, "aggregate": k * P, "stats": N * P}
-    peak, peak_kind = measured_peak()
-    kernels = {}
+    kernels = {"round": {"avg_ms": round_ms, "algorithmic_bytes": round_bytes,
+                         "achieved_gbs": round_gbs, frac_key: round_gbs / peak,
+                         "frac_of_8TBs": round_gbs / 8000.0, "mean_steps_per_device": mean_steps,
+                         "gelem_steps_per_s": N * P * mean_steps / (round_ms * 1e-3) / 1e9,
+                         "traffic": None if NCU_DRAM_BYTES_PER_ELEM["round"] is None
+                         else NCU_DRAM_BYTES_PER_ELEM["round"] * N * P}}
     for n in names:
         gbs = alg_bytes[n] / (kern_ms[n] * 1e-3) / 1e9
         per_elem = NCU_DRAM_BYTES_PER_ELEM[n]
         kernels[n] = {"avg_ms": kern_ms[n], "algorithmic_bytes": alg_bytes[n], "achieved_gbs": gbs,
-                      "frac_of_%s_hbm" % peak_kind: gbs / peak, "frac_of_8TBs": gbs / 8000.0,
-                      "share_of_step": kern_ms[n] / (elapsed_ms / K),
+                      frac_key: gbs / peak, "frac_of_8TBs": gbs / 8000.0,
+                      "share_of_separate_round": kern_ms[n] / sep_ms,
                       "traffic": None if per_elem is None else per_elem * units[n]}
-    kernels["local_step"]["mean_steps_per_device"] = mean_steps
-    kernels["local_step"]["gelem_steps_per_s"] = N * P * mean_steps / (kern_ms["local_step"] * 1e-3) / 1e9
-    dominant = max(names, key=lambda n: kern_ms[n])
-    roofline = {"kernel": dominant, "bound": "hbm", "achieved": kernels[dominant]["achieved_gbs"],
-                "peak": peak, "unit": "GB/s", "frac": kernels[dominant]["achieved_gbs"] / peak,
-                "peak_source": "of measured (copy bandwidth of this pool's B200s)"
-                if peak_kind == "measured" else "of fallback (6650 GB/s)",
-                "traffic": kernels[dominant]["traffic"]}
-    if dominant == "local_step":
-        roofline["note"] = ("bytes per launch do not depend on the step count; at a mean of %.2f "
-                            "steps per device the kernel is limited by generator arithmetic "
-                            "(integer multiply + special-function units), not by HBM" % mean_steps)
+    kernels["local_step"]["mean_steps_per_device"] = sep_mean_steps
+    kernels["local_step"]["gelem_steps_per_s"] = N * P * sep_mean_steps / (kern_ms["local_step"] * 1e-3) / 1e9
+    separate = {"rounds_per_s": world * 1e3 / sep_ms, "ms_per_round": sep_ms, "rounds": Ks,
+                "what": "hadfl_local_step + hadfl_select + hadfl_aggregate + hadfl_stats_enqueue"}
+    alu_peak = SM_COUNT * LANES_PER_CLK_PER_SM * SM_MAX_GHZ / ALU_INSTR_PER_ELEM_STEP   # Gelem-step/s
+    alu_achieved = kernels["round"]["gelem_steps_per_s"]
+    hbm_src = ("of measured (copy bandwidth of this pool's B200s)" if peak_kind == "measured"
+               else "of fallback (6650 GB/s)")
+    # which floor is higher for this launch: bytes / HBM peak or element-steps / issue peak?
+    t_hbm, t_alu = round_bytes / (peak * 1e9), N * P * mean_steps / (alu_peak * 1e9)
+    if t_alu > t_hbm:
+        roofline = {"kernel": "k_round (the whole round in one launch)", "bound": "alu",
+                    "achieved": alu_achieved, "peak": alu_peak, "unit": "Gelem-step/s",
+                    "frac": alu_achieved / alu_peak,
+                    "peak_source": "derived: 148 SMs x 128 lane-instr/clk x 1.965 GHz / 20.5 "
+                                   "instructions per parameter and step (instruction issue)",
+                    "hbm_achieved_gbs": round_gbs, "hbm_peak_gbs": peak,
+                    "hbm_frac": round_gbs / peak, "hbm_peak_source": hbm_src}
+    else:
+        roofline = {"kernel": "k_round (the whole round in one launch)", "bound": "hbm",
+                    "achieved": round_gbs, "peak": peak, "unit": "GB/s", "frac": round_gbs / peak,
+                    "peak_source": hbm_src, "alu_achieved_gelem_steps": alu_achieved,
+                    "alu_peak_gelem_steps": alu_peak, "alu_frac": alu_achieved / alu_peak}
+    roofline["traffic"] = kernels["round"]["traffic"]
+    roofline["note"] = ("algorithmic bytes = 16 per (device, parameter) whatever the step count; "
+                        "mean steps per device here: %.2f; the bandwidth-bound kernels (local update "
+                        "at 1 step, aggregation, statistics) are listed under `kernels`" % mean_steps)
 
     # ---- end to end: host buffers, results read back every round -----------------------------
     Ke = max(3, min(K, 200))
@@ -288,7 +341,7 @@ def run_ours(args, wl):
     barrier()
     t0 = time.perf_counter()
     for i in range(Ke):
-        sel = arena.run_round(r + i)
+        sel = arena.run_round_fused(r + i)
         n2, d2 = h.stats_read()
         h.read_params(int(sel[0]), out=host_model)
     torch.cuda.synchronize()
@@ -298,14 +351,14 @@ def run_ours(args, wl):
     d2h = 2 * N * 4 + P * 4                    # statistics + the aggregated model
     e2e = {"value": world * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": Ke,
-           "what": "round + hadfl_stats_read + hadfl_read_params(selected[0]) into pinned host memory"}
+           "what": "hadfl_round + hadfl_stats_read + hadfl_read_params(selected[0]) into pinned host memory"}
 
     line = {"metric": METRIC, "value": world * K / (elapsed_ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": warmup,
             "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": describe(wl),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "kernels": kernels}
+            "kernels": kernels, "separate_calls": separate}
 
     arena.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
