@@ -151,14 +151,79 @@ __device__ __forceinline__ void st_pack(__nv_bfloat16 *row, int64_t p, const flo
     *reinterpret_cast<uint2 *>(row + 4 * p) = raw;
   }
 }
-template <typename T, int E>
-__device__ __forceinline__ void ld_pack_any(const T *row, int64_t p, int live, float (&v)[E]) {
+// A loaded pack as it came from memory.  Loads fill a RawPack and nothing else, so that a thread
+// can issue all the loads of a batch (or the prefetch of the next row) without an instruction that
+// depends on the data in between; `unpack` widens to fp32 registers at the point of use.
+template <typename WT, int E>
+struct RawPack;
+template <int E>
+struct RawPack<float, E> {
+  float v[E];
+};
+template <>
+struct RawPack<__nv_bfloat16, 8> {
+  uint4 q;
+};
+template <>
+struct RawPack<__nv_bfloat16, 4> {
+  uint2 q;
+};
+
+template <int E>
+__device__ __forceinline__ void unpack(const RawPack<float, E> &r, float (&v)[E]) {
+#pragma unroll
+  for (int i = 0; i < E; ++i) v[i] = r.v[i];
+}
+__device__ __forceinline__ void unpack(const RawPack<__nv_bfloat16, 8> &r, float (&v)[8]) {
+  bf16x2_to_floats(r.q.x, v[0], v[1]);
+  bf16x2_to_floats(r.q.y, v[2], v[3]);
+  bf16x2_to_floats(r.q.z, v[4], v[5]);
+  bf16x2_to_floats(r.q.w, v[6], v[7]);
+}
+__device__ __forceinline__ void unpack(const RawPack<__nv_bfloat16, 4> &r, float (&v)[4]) {
+  bf16x2_to_floats(r.q.x, v[0], v[1]);
+  bf16x2_to_floats(r.q.y, v[2], v[3]);
+}
+
+// `at` points to the first element of the pack.  live == E: vector load; otherwise (the ragged
+// last pack of a row) element by element, dead lanes read as 0.
+template <int E>
+__device__ __forceinline__ void ld_raw(const float *at, int live, RawPack<float, E> &r) {
   if (live == E) {
-    ld_pack<E>(row, p, v);
+#pragma unroll
+    for (int i = 0; i < E / 4; ++i) {
+      const float4 t = *reinterpret_cast<const float4 *>(at + 4 * i);
+      r.v[4 * i] = t.x; r.v[4 * i + 1] = t.y; r.v[4 * i + 2] = t.z; r.v[4 * i + 3] = t.w;
+    }
   } else {
 #pragma unroll
-    for (int i = 0; i < E; ++i) v[i] = i < live ? ld_elem(row, E * p + i) : 0.f;
+    for (int i = 0; i < E; ++i) r.v[i] = i < live ? at[i] : 0.f;
   }
+}
+__device__ __forceinline__ uint32_t ld_bf16_bits(const __nv_bfloat16 *at, int i, int live) {
+  return i < live ? (uint32_t)*reinterpret_cast<const unsigned short *>(at + i) : 0u;
+}
+__device__ __forceinline__ void ld_raw(const __nv_bfloat16 *at, int live, RawPack<__nv_bfloat16, 8> &r) {
+  if (live == 8) {
+    r.q = *reinterpret_cast<const uint4 *>(at);
+  } else {
+    r.q.x = ld_bf16_bits(at, 0, live) | (ld_bf16_bits(at, 1, live) << 16);
+    r.q.y = ld_bf16_bits(at, 2, live) | (ld_bf16_bits(at, 3, live) << 16);
+    r.q.z = ld_bf16_bits(at, 4, live) | (ld_bf16_bits(at, 5, live) << 16);
+    r.q.w = ld_bf16_bits(at, 6, live) | (ld_bf16_bits(at, 7, live) << 16);
+  }
+}
+__device__ __forceinline__ void ld_raw(const __nv_bfloat16 *at, int live, RawPack<__nv_bfloat16, 4> &r) {
+  if (live == 4) {
+    r.q = *reinterpret_cast<const uint2 *>(at);
+  } else {
+    r.q.x = ld_bf16_bits(at, 0, live) | (ld_bf16_bits(at, 1, live) << 16);
+    r.q.y = ld_bf16_bits(at, 2, live) | (ld_bf16_bits(at, 3, live) << 16);
+  }
+}
+template <typename WT, int E>
+__device__ __forceinline__ void zero_raw(RawPack<WT, E> &r) {
+  memset(&r, 0, sizeof(r));
 }
 template <typename T, int E>
 __device__ __forceinline__ void st_pack_any(T *row, int64_t p, int live, const float (&v)[E]) {
@@ -398,18 +463,29 @@ k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalS
   char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
   char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(float));
 
-  auto load = [&](int j, float (&wv)[E], float (&mv)[E]) {
-    ld_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-    ld_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+  auto load = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+    ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+    ld_raw(at_row<float>(mp, a.r[j].m_off), live, rm);
   };
-  auto visit = [&](int j, float (&wv)[E], float (&mv)[E]) {
+  auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
+    sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+    st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+    st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+  };
+  // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
+  auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
     if (a.r[j].steps > 0) {
-      sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-      st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-      st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+      if constexpr (sizeof(WT) == 4) {
+        body(j, rw.v, rm.v);
+      } else {
+        float wv[E];
+        unpack(rw, wv);
+        body(j, wv, rm.v);
+      }
     }
   };
-  float w0[E], m0[E], w1[E], m1[E];
+  RawPack<WT, E> w0, w1;
+  RawPack<float, E> m0, m1;
   load(0, w0, m0);
   int j = 0;
   for (; j + 1 < a.n; j += 2) {
@@ -442,27 +518,29 @@ template <typename WT, int KR, int E>
 __device__ __forceinline__ void combine_pack(const WT *__restrict__ w, int64_t stride,
                                              const CombineArgs &c, int64_t p, int live,
                                              float (&acc)[E]) {
-  constexpr int B = KR > 0 ? (KR * E <= 64 ? KR : 64 / E) : 32 / E;
+  constexpr int B = KR > 0 ? (KR <= 16 ? KR : 16) : 8;  // rows per batch: at most 16 x 16 bytes in registers
   const int nr = KR > 0 ? KR : c.nr;
 #pragma unroll
   for (int i = 0; i < E; ++i) acc[i] = 0.f;
 #pragma unroll
   for (int base = 0; base < (KR > 0 ? KR : kMaxDevices); base += B) {
     if (base >= nr) break;
-    float v[B][E];
+    RawPack<WT, E> raw[B];
 #pragma unroll
     for (int j = 0; j < B; ++j)
-      if (base + j < nr) ld_pack_any(w + (int64_t)c.rd[base + j] * stride, p, live, v[j]);
+      if (base + j < nr) ld_raw(w + (int64_t)c.rd[base + j] * stride + (int64_t)E * p, live, raw[j]);
 #pragma unroll
     for (int j = 0; j < B; ++j) {
       if (base + j < nr) {
         const float aj = c.a[base + j];
+        float v[E];
+        unpack(raw[j], v);
         if (base + j == 0) {
 #pragma unroll
-          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(aj, v[j][i]);
+          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(aj, v[i]);
         } else {
 #pragma unroll
-          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, v[j][i], acc[i]);
+          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, v[i], acc[i]);
         }
       }
     }
@@ -568,26 +646,29 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
   double n2 = 0.0, d2 = 0.0;
   for (int64_t chunk = my_lane; chunk < n_chunks; chunk += lanes) {
     const int64_t p0 = chunk * per_chunk + threadIdx.x;
-    float v[U][E], r[U][E];
+    RawPack<WT, E> rv[U], rr[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int64_t p = p0 + (int64_t)u * kThreads;
       const int live = live_of(n_params, p, E);
       if (live > 0) {
-        ld_pack_any(my_row, p, live, v[u]);
-        ld_pack_any(ref_row, p, live, r[u]);
+        ld_raw(my_row + (int64_t)E * p, live, rv[u]);
+        ld_raw(ref_row + (int64_t)E * p, live, rr[u]);
       } else {
-#pragma unroll
-        for (int i = 0; i < E; ++i) v[u][i] = r[u][i] = 0.f;
+        zero_raw(rv[u]);
+        zero_raw(rr[u]);
       }
     }
     float a = 0.f, b = 0.f;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
+      float v[E], r[E];
+      unpack(rv[u], v);
+      unpack(rr[u], r);
 #pragma unroll
       for (int i = 0; i < E; ++i) {
-        const float d = v[u][i] - r[u][i];
-        a = fmaf(v[u][i], v[u][i], a);
+        const float d = v[i] - r[i];
+        a = fmaf(v[i], v[i], a);
         b = fmaf(d, d, b);
       }
     }
@@ -676,14 +757,14 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
 #pragma unroll
     for (int i = 0; i < E; ++i) acc[i] = 0.f;
 
-    auto load = [&](int j, float (&wv)[E], float (&mv)[E]) {
+    auto load = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
       if (act) {
-        ld_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-        if (a.r[j].steps > 0) ld_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+        if (a.r[j].steps > 0) ld_raw(at_row<float>(mp, a.r[j].m_off), live, rm);
       }
     };
     // One row: its steps, then its part in the aggregation / synchronisation and in the sums.
-    auto visit = [&](int j, float (&wv)[E], float (&mv)[E]) {
+    auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
       const bool stepped = act && a.r[j].steps > 0;
       if (stepped) {
         sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
@@ -728,9 +809,22 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
         add_row_sums(s_acc, j, n2, d2, lane);
       }
     };
-    float w0[E], m0[E], w1[E], m1[E];
-#pragma unroll
-    for (int i = 0; i < E; ++i) w0[i] = m0[i] = w1[i] = m1[i] = 0.f;
+    // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
+    auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+      if constexpr (sizeof(WT) == 4) {
+        body(j, rw.v, rm.v);
+      } else {
+        float wv[E];
+        unpack(rw, wv);
+        body(j, wv, rm.v);
+      }
+    };
+    RawPack<WT, E> w0, w1;
+    RawPack<float, E> m0, m1;
+    zero_raw(w0);
+    zero_raw(w1);
+    zero_raw(m0);
+    zero_raw(m1);
     load(0, w0, m0);
     int j = 0;
     for (; j + 1 < a.n; j += 2) {
