@@ -126,3 +126,21 @@ def test_c5_bandwidth_sweep_sizes(oracle, log2_p, dtype):
 def test_c5_smallest_size_full_arena_first_rounds(oracle, dtype):
     wl = workloads.shrink(workloads.c5(16, dtype=dtype, hetero=True), 1 << 16, rounds=5)
     run_and_compare(oracle, wl, None, check_rounds=range(5), stats_rounds=range(5))
+
+
+def test_rows_longer_than_two_to_the_31_elements(oracle):
+    """Index arithmetic beyond 32 bits: two replicas of 2^31 + 6 parameters (row byte offsets and
+    element indices above 2^32; column-group indices above 2^29), checked on sampled columns,
+    through the separate calls and through the fused round."""
+    from paper_2111_08274_b200.workloads import Workload
+    P = 2**31 + 6
+    wl = Workload("huge", 2, P, 2, 2, "fixed", (2, 1), grad_std=1e-2, seed=workloads.BASE_SEED + 99)
+    groups = workloads.sample_groups(P, 512, 256, seed=7)
+    run_and_compare(oracle, wl, groups, check_rounds=(0,))
+    arena = runtime.Arena(wl)
+    sim = make_sim(oracle, wl, groups)
+    for r in range(wl.rounds):
+        sel = arena.run_round_fused(r)
+        assert np.array_equal(sel, oracle_round(sim, wl, r))
+    compare_sample(arena, sim, groups, "huge fused")
+    arena.close()
