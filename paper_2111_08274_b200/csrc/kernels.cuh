@@ -552,6 +552,34 @@ __global__ void __launch_bounds__(kThreads)
 k_combine(WT *__restrict__ w, int64_t stride, int64_t n_params, CombineArgs c) {
   constexpr int E = Pack16<WT>::E;
   const int64_t p0 = (int64_t)blockIdx.x * (kThreads * U) + threadIdx.x;
+  // Fast path (all but the last block of a launch): every pack of the block is full, so the
+  // U * KR row loads of a thread are straight-line code and all in flight together.
+  const bool block_full = ((int64_t)(blockIdx.x + 1) * (kThreads * U)) * E <= n_params;
+  if (KR > 0 && KR * U <= 16 && block_full) {
+    constexpr int KRc = KR > 0 ? KR : 1;
+    RawPack<WT, E> raw[U][KRc];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int j = 0; j < KRc; ++j)
+        ld_raw(w + (int64_t)c.rd[j] * stride + (int64_t)E * (p0 + (int64_t)u * kThreads), E, raw[u][j]);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float acc[E], v[E];
+      unpack(raw[u][0], v);
+#pragma unroll
+      for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(c.a[0], v[i]);
+#pragma unroll
+      for (int j = 1; j < KRc; ++j) {
+        unpack(raw[u][j], v);
+#pragma unroll
+        for (int i = 0; i < E; ++i) acc[i] = fmaf(c.a[j], v[i], acc[i]);
+      }
+      for (int j = 0; j < c.nw; ++j)
+        st_pack<E>(w + (int64_t)c.wr[j] * stride, p0 + (int64_t)u * kThreads, acc);
+    }
+    return;
+  }
   float acc[U][E];
   int live[U];
 #pragma unroll
@@ -647,16 +675,24 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
   for (int64_t chunk = my_lane; chunk < n_chunks; chunk += lanes) {
     const int64_t p0 = chunk * per_chunk + threadIdx.x;
     RawPack<WT, E> rv[U], rr[U];
+    if ((chunk + 1) * per_chunk * E <= n_params) {  // every pack of the chunk is full: no branches
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int64_t p = p0 + (int64_t)u * kThreads;
-      const int live = live_of(n_params, p, E);
-      if (live > 0) {
-        ld_raw(my_row + (int64_t)E * p, live, rv[u]);
-        ld_raw(ref_row + (int64_t)E * p, live, rr[u]);
-      } else {
-        zero_raw(rv[u]);
-        zero_raw(rr[u]);
+      for (int u = 0; u < U; ++u) {
+        ld_raw(my_row + (int64_t)E * (p0 + (int64_t)u * kThreads), E, rv[u]);
+        ld_raw(ref_row + (int64_t)E * (p0 + (int64_t)u * kThreads), E, rr[u]);
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int64_t p = p0 + (int64_t)u * kThreads;
+        const int live = live_of(n_params, p, E);
+        if (live > 0) {
+          ld_raw(my_row + (int64_t)E * p, live, rv[u]);
+          ld_raw(ref_row + (int64_t)E * p, live, rr[u]);
+        } else {
+          zero_raw(rv[u]);
+          zero_raw(rr[u]);
+        }
       }
     }
     float a = 0.f, b = 0.f;
