@@ -1,18 +1,20 @@
 // sm_100a kernels of the HADFL round: initial model (K0), batched heterogeneity-aware local
-// update (K1; Eq. 3 / Algorithm 1), fused weighted aggregation with write-back (K2; Eq. 5), and
-// per-replica statistics (K3).
+// update (K1; Eq. 3 / Algorithm 1), fused weighted aggregation with write-back (K2; Eq. 5),
+// per-replica statistics (K3), and the fused round (K1 + K2 + global synchronisation + K3 in one
+// pass over the arena).
 //
-// All of them stream rows of one [N][stride] arena.  The unit of work is a "column group": four
-// consecutive parameters, one 128-bit access for fp32 storage (64-bit for bf16 storage) and one
-// Philox block.  In K1 and K2 a thread owns a column group and walks over the rows, so that
-//   - accesses of a warp are 512 contiguous bytes per row,
-//   - several independent row loads are in flight per thread before the first dependent use,
+// All of them stream rows of one [N][stride] arena.  A "column group" is four consecutive
+// parameters (one Philox block); a thread holds a "pack" of a row - 16 bytes of w in K2 / K3,
+// eight parameters in K1 and the fused round - and walks over the rows, so that
+//   - accesses of a warp are contiguous (512 bytes per 128-bit load instruction),
+//   - several independent row loads are in flight per thread before the first dependent use
+//     (loads fill raw packs; widening bf16 to fp32 happens where the values are used),
 //   - every thread does the same amount of arithmetic whatever the per-device step counts are
 //     (the kernel-level answer to the straggler problem the paper is about), and
 //   - the arithmetic order per element is fixed, hence results are reproducible bit for bit.
 // None of this is a dense contraction, so there is no tensor-core path: the bound is HBM
-// bandwidth, except for K1 with many steps per device, where the integer multiplies of Philox
-// and the special-function unit (log2, sqrt, sin, cos) bind.
+// bandwidth, except for the local update with several steps per device, where instruction issue
+// (the integer multiplies of Philox, Box-Muller on the special-function unit) binds.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -26,24 +28,11 @@ constexpr int kMaxDevices = 32;
 constexpr int kThreads = 256;
 
 // ------------------------------------------------------------------------------------------
-// Storage access: a column group of fp32 or bf16 parameters <-> four fp32 registers.
-// `live` is the number of lanes of the group that are parameters (4 except in a ragged last
-// group); dead lanes read as 0 and are never written.
+// Storage access by element and by column group (used by the initial-model kernel and by the
+// ragged last pack of a row).
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ float4 ld_group(const float *row, int64_t g) {
-  return *reinterpret_cast<const float4 *>(row + 4 * g);
-}
 __device__ __forceinline__ void st_group(float *row, int64_t g, float4 v) {
   *reinterpret_cast<float4 *>(row + 4 * g) = v;
-}
-__device__ __forceinline__ float4 ld_group(const __nv_bfloat16 *row, int64_t g) {
-  const uint2 raw = *reinterpret_cast<const uint2 *>(row + 4 * g);
-  float4 v;
-  v.x = __uint_as_float(raw.x << 16);
-  v.y = __uint_as_float(raw.x & 0xFFFF0000u);
-  v.z = __uint_as_float(raw.y << 16);
-  v.w = __uint_as_float(raw.y & 0xFFFF0000u);
-  return v;
 }
 __device__ __forceinline__ void st_group(__nv_bfloat16 *row, int64_t g, float4 v) {
   const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
@@ -62,32 +51,6 @@ __device__ __forceinline__ void st_elem(__nv_bfloat16 *row, int64_t p, float v) 
   row[p] = __float2bfloat16_rn(v);
 }
 
-template <typename T>
-__device__ __forceinline__ float4 ld_group_ragged(const T *row, int64_t g, int live) {
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (live > 0) v.x = ld_elem(row, 4 * g + 0);
-  if (live > 1) v.y = ld_elem(row, 4 * g + 1);
-  if (live > 2) v.z = ld_elem(row, 4 * g + 2);
-  return v;
-}
-template <typename T>
-__device__ __forceinline__ void st_group_ragged(T *row, int64_t g, int live, float4 v) {
-  if (live > 0) st_elem(row, 4 * g + 0, v.x);
-  if (live > 1) st_elem(row, 4 * g + 1, v.y);
-  if (live > 2) st_elem(row, 4 * g + 2, v.z);
-}
-template <typename T>
-__device__ __forceinline__ float4 ld_any(const T *row, int64_t g, int live) {
-  return live == 4 ? ld_group(row, g) : ld_group_ragged(row, g, live);
-}
-template <typename T>
-__device__ __forceinline__ void st_any(T *row, int64_t g, int live, float4 v) {
-  if (live == 4)
-    st_group(row, g, v);
-  else
-    st_group_ragged(row, g, live, v);
-}
-
 // ------------------------------------------------------------------------------------------
 // Packs: E consecutive parameters held by one thread (E = 4 or 8).  fp32: E/4 128-bit accesses;
 // bf16: one 64-bit (E = 4) or 128-bit (E = 8) access.  A pack of 8 is two column groups, i.e.
@@ -98,14 +61,6 @@ struct Pack16 {  // the pack that is 16 bytes of storage
   static constexpr int E = sizeof(WT) == 2 ? 8 : 4;
 };
 
-template <int E>
-__device__ __forceinline__ void ld_pack(const float *row, int64_t p, float (&v)[E]) {
-#pragma unroll
-  for (int i = 0; i < E / 4; ++i) {
-    const float4 t = *reinterpret_cast<const float4 *>(row + E * p + 4 * i);
-    v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
-  }
-}
 template <int E>
 __device__ __forceinline__ void st_pack(float *row, int64_t p, const float (&v)[E]) {
 #pragma unroll
@@ -120,20 +75,6 @@ __device__ __forceinline__ void bf16x2_to_floats(uint32_t raw, float &lo, float 
 __device__ __forceinline__ uint32_t floats_to_bf16x2(float lo, float hi) {
   const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t *>(&t);
-}
-template <int E>
-__device__ __forceinline__ void ld_pack(const __nv_bfloat16 *row, int64_t p, float (&v)[E]) {
-  if (E == 8) {
-    const uint4 raw = *reinterpret_cast<const uint4 *>(row + 8 * p);
-    bf16x2_to_floats(raw.x, v[0], v[1]);
-    bf16x2_to_floats(raw.y, v[2], v[3]);
-    bf16x2_to_floats(raw.z, v[E - 4], v[E - 3]);
-    bf16x2_to_floats(raw.w, v[E - 2], v[E - 1]);
-  } else {
-    const uint2 raw = *reinterpret_cast<const uint2 *>(row + 4 * p);
-    bf16x2_to_floats(raw.x, v[0], v[1]);
-    bf16x2_to_floats(raw.y, v[2], v[3]);
-  }
 }
 template <int E>
 __device__ __forceinline__ void st_pack(__nv_bfloat16 *row, int64_t p, const float (&v)[E]) {
@@ -605,19 +546,6 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
-// Sums two per-lane values over the warp with five shuffles: after the first exchange the lower
-// half-warp carries `a` and the upper half carries `b`.  Lane 0 ends with sum(a), lane 16 with
-// sum(b); the order of additions is fixed.
-__device__ __forceinline__ float warp_sum_pair(float a, float b, int lane) {
-  const bool upper = (lane & 16) != 0;
-  float mine = upper ? b : a;
-  const float give = upper ? a : b;
-  mine += __shfl_xor_sync(0xFFFFFFFFu, give, 16);
-#pragma unroll
-  for (int off = 8; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
-  return mine;
-}
-
 // Last-block finish: the block that draws the last ticket sums partials[t][0 .. n_src) for every
 // t < n_vals in a fixed order (a warp per value, lanes strided, then the butterfly), hands the
 // sums to `emit`, and resets the ticket.  Returns without waiting for anyone.
@@ -766,7 +694,7 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
 }
 
 template <typename WT, typename Gen, int E>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
         StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
@@ -855,21 +783,16 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
         body(j, wv, rm.v);
       }
     };
-    RawPack<WT, E> w0, w1;
-    RawPack<float, E> m0, m1;
-    zero_raw(w0);
-    zero_raw(w1);
-    zero_raw(m0);
-    zero_raw(m1);
-    load(0, w0, m0);
-    int j = 0;
-    for (; j + 1 < a.n; j += 2) {
-      load(j + 1, w1, m1);
-      visit(j, w0, m0);
-      if (j + 2 < a.n) load(j + 2, w0, m0);
-      visit(j + 1, w1, m1);
+    // No prefetch of the next row here (unlike K1): the registers it would take cost a resident
+    // block, and three blocks per SM hide the row loads better than two blocks with a prefetch.
+    RawPack<WT, E> rw;
+    RawPack<float, E> rm;
+    zero_raw(rw);
+    zero_raw(rm);
+    for (int j = 0; j < a.n; ++j) {
+      load(j, rw, rm);
+      visit(j, rw, rm);
     }
-    if (j < a.n) visit(j, w0, m0);
   }
   // ---- block: fold the per-thread slots (lower half-warps hold norms, upper halves distances)
   for (int j = a.k - 1; j < a.n; ++j) {
