@@ -233,15 +233,23 @@ struct NormalsFast {
   // Next to u0 = 1 (x0 >= 2^32 - 2^22) lg2.approx only has an absolute error bound, so the exact
   // complement and a series take over.  Measured against a double-precision evaluation (s = 1):
   // max |dz| about 2e-6, mean 1.6e-7.
-  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float lg_scale,
-                                              float scale2, float &z0, float &z1) {
-    const float u0 = fmaf(__uint2float_rn(x0), 0x1p-32f, 0x1p-33f);
-    float r2 = lg_scale * sfu_lg2(u0);
-    if (x0 >= 0xFFC00000u) r2 = r2_next_to_one(x0, scale2);
+  static constexpr uint32_t kNearOne = 0xFFC00000u;
+  // r^2 away from u0 = 1 (wrong by up to a few 1e-7 absolute next to it: see needs_series)
+  static __device__ __forceinline__ float radius2(uint32_t x0, float lg_scale) {
+    return lg_scale * sfu_lg2(fmaf(__uint2float_rn(x0), 0x1p-32f, 0x1p-33f));
+  }
+  static __device__ __forceinline__ bool needs_series(uint32_t x0) { return x0 >= kNearOne; }
+  static __device__ __forceinline__ void finish(float r2, uint32_t x1, float &z0, float &z1) {
     const float theta = fmaf(__int2float_rn((int)x1), 1.4629180792671596e-9f, 7.314590396335798e-10f);
     const float r = sfu_sqrt(r2);
     z0 = r * sfu_cos(theta);
     z1 = r * sfu_sin(theta);
+  }
+  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float lg_scale,
+                                              float scale2, float &z0, float &z1) {
+    float r2 = radius2(x0, lg_scale);
+    if (needs_series(x0)) r2 = r2_next_to_one(x0, scale2);
+    finish(r2, x1, z0, z1);
   }
 };
 
@@ -358,6 +366,10 @@ struct GroupProducts {
   }
 };
 
+// The steps of one device on one pack.  Each step is written stage by stage over all NB Philox
+// blocks of the pack - all generator rounds, then all radii, one combined test for the rare
+// "u0 next to 1" case, then all angles, then the update - so that the independent chains sit in
+// the same straight-line code and the hardware scheduler can interleave them.
 template <typename Gen, int NB>
 __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB],
                                           const GroupProducts<NB> &gp, const RowStep &rs,
@@ -367,14 +379,35 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
   for (int b = 0; b < NB; ++b) c2_first[b] = gp.hi[b] ^ rs.r1_c2;
   for (int e = 0; e < rs.steps; ++e) {
     const uint32_t c0_first = rs.r1_c0 ^ (rs.base_lo + (uint32_t)e);
+    uint32_t x[NB][4];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      uint32_t c0 = c0_first, c1 = rs.r1_c1, c2 = c2_first[b], c3 = gp.lo[b];
+      x[b][0] = c0_first; x[b][1] = rs.r1_c1; x[b][2] = c2_first[b]; x[b][3] = gp.lo[b];
+    }
 #pragma unroll
-      for (int r = 1; r < 10; ++r) philox_round(c0, c1, c2, c3, keys.a[r], keys.b[r]);
+    for (int r = 1; r < 10; ++r)
+#pragma unroll
+      for (int b = 0; b < NB; ++b) philox_round(x[b][0], x[b][1], x[b][2], x[b][3], keys.a[r], keys.b[r]);
+    float r2[NB][2];
+    uint32_t top = 0;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      r2[b][0] = Gen::radius2(x[b][0], k.lg_scale);
+      r2[b][1] = Gen::radius2(x[b][2], k.lg_scale);
+      top = max(top, max(x[b][0], x[b][2]));
+    }
+    if (Gen::needs_series(top)) {  // about once in 250 steps of a pack
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+        if (Gen::needs_series(x[b][0])) r2[b][0] = r2_next_to_one(x[b][0], k.scale2);
+        if (Gen::needs_series(x[b][2])) r2[b][1] = r2_next_to_one(x[b][2], k.scale2);
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
       float n[4];  // grad_std * z
-      Gen::pair(c0, c1, k.lg_scale, k.scale2, n[0], n[1]);
-      Gen::pair(c2, c3, k.lg_scale, k.scale2, n[2], n[3]);
+      Gen::finish(r2[b][0], x[b][1], n[0], n[1]);
+      Gen::finish(r2[b][1], x[b][3], n[2], n[3]);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float g = fmaf(k.wd, w[4 * b + i], n[i]);
