@@ -43,10 +43,11 @@ METRIC = "aggregation_rounds_per_sec"
 UNIT = "rounds/s"
 FALLBACK_HBM_GBS = 6650.0
 # Arithmetic roofline of the local update: instruction issue.  One step of one Philox block
-# (4 parameters) needs at least 82 warp instructions (9 Philox rounds x (2 wide multiplies +
-# 2 three-input xors) = 36, Box-Muller for two pairs = 28, the update = 12, step loop = 6), i.e.
-# 20.5 per parameter and step; an SM issues 4 x 32 = 128 lane-instructions per clock.
-ALU_INSTR_PER_ELEM_STEP = 20.5
+# (4 parameters) needs at least 76 warp instructions (9 Philox rounds x (2 wide multiplies +
+# 2 three-input xors) = 36, Box-Muller for two pairs = 24, the rare-case test = 2, the update = 12,
+# step loop = 2), i.e. 19 per parameter and step (ncu counts 78 in the kernel as it stands); an
+# SM issues 4 x 32 = 128 lane-instructions per clock.
+ALU_INSTR_PER_ELEM_STEP = 19.0
 SM_COUNT, LANES_PER_CLK_PER_SM, SM_MAX_GHZ = 148, 128, 1.965
 ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to size its sample
 
@@ -54,7 +55,7 @@ ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to 
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same kernel;
 # reads grow in proportion to the elements processed; writes are undercounted by whatever is still
 # dirty in the 126 MB L2 when the kernel ends).  None = not captured for the kernel as it stands.
-NCU_DRAM_BYTES_PER_ELEM = {"round": 14.24, "local_step": 14.28, "aggregate": 4.54, "stats": 4.11}
+NCU_DRAM_BYTES_PER_ELEM = {"round": 14.25, "local_step": 14.29, "aggregate": 4.52, "stats": 4.12}
 
 
 def measured_peak():
@@ -321,7 +322,7 @@ def run_ours(args, wl):
         roofline = {"kernel": "k_round (the whole round in one launch)", "bound": "alu",
                     "achieved": alu_achieved, "peak": alu_peak, "unit": "Gelem-step/s",
                     "frac": alu_achieved / alu_peak,
-                    "peak_source": "derived: 148 SMs x 128 lane-instr/clk x 1.965 GHz / 20.5 "
+                    "peak_source": "derived: 148 SMs x 128 lane-instr/clk x 1.965 GHz / 19 "
                                    "instructions per parameter and step (instruction issue)",
                     "hbm_achieved_gbs": round_gbs, "hbm_peak_gbs": peak,
                     "hbm_frac": round_gbs / peak, "hbm_peak_source": hbm_src}
