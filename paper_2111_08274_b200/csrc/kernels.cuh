@@ -426,8 +426,11 @@ __device__ __forceinline__ WT *at_row(char *pack_in_row0, int64_t row_off) {
   return reinterpret_cast<WT *>(pack_in_row0 + row_off);
 }
 
-template <typename WT, typename Gen, int E>
-__global__ void __launch_bounds__(kThreads)
+// MINB: resident blocks per SM the register allocation must allow.  With bf16 storage and few
+// steps per device the launch is bandwidth-bound and gains from a fourth resident block (64
+// registers); with many steps the unconstrained allocation is faster.  The host picks.
+template <typename WT, typename Gen, int E, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalStepArgs a,
              PhiloxKeys keys, StepConsts k) {
   const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
