@@ -342,3 +342,26 @@ def test_checkpoint_resume_is_exact():
     for i in range(3):
         assert np.array_equal(a.read_params(i), b.read_params(i))
         assert np.array_equal(a.read_momentum(i), b.read_momentum(i))
+
+
+def test_state_errors():
+    """Calls that are not valid in the handle's state say so and change nothing."""
+    wl = small(2, 1000)
+    h = gpu(wl)
+    with pytest.raises(binding.HadflError) as e:
+        h.stats_read()                      # nothing enqueued yet
+    assert e.value.code == binding.ERR_STATE
+    h.set_versions(step_counts=np.array([2**56 - 3, 0], dtype=np.uint64))
+    before = h.read_params(0)
+    with pytest.raises(binding.HadflError) as e:
+        h.local_step([0, 1], [4, 1], 0.01)  # device 0's gradient stream would run past 2^56 steps
+    assert e.value.code == binding.ERR_STATE
+    with pytest.raises(binding.HadflError) as e:
+        h.round([0, 1], [4, 1], 0.01, 0, 1, 3)
+    assert e.value.code == binding.ERR_STATE
+    with pytest.raises(binding.HadflError):
+        h.set_versions(step_counts=np.array([2**56, 0], dtype=np.uint64))
+    assert np.array_equal(h.read_params(0), before)
+    assert list(h.get_versions()[1]) == [2**56 - 3, 0]
+    h.local_step([0, 1], [2, 1], 0.01)      # up to the limit is fine
+    assert list(h.get_versions()[1]) == [2**56 - 1, 1]
