@@ -206,6 +206,18 @@ int hadfl_read_momentum(hadfl_handle *h, int32_t device_id, float *dst, int64_t 
 int hadfl_write_params(hadfl_handle *h, int32_t device_id, const float *src, int64_t count);
 int hadfl_write_momentum(hadfl_handle *h, int32_t device_id, const float *src, int64_t count);
 
+/* Model backup that overlaps with the rounds that follow (Section "Overall Design", item 9: the model
+ * manager "regularly fetches the latest model").  hadfl_backup_begin takes a snapshot of the first
+ * `count` parameters of device_id as they are at this point of the handle's stream (one device-to-
+ * device copy on that stream into a staging row the library allocates on first use) and then moves
+ * it to `dst` on a separate copy stream: the caller and the later work on the handle's stream do not
+ * wait for the transfer.  dst (fp32, widened from bf16 storage) must stay valid until
+ * hadfl_backup_wait returns, which blocks until the data has arrived; use pinned host memory for the
+ * copy to be asynchronous.  One backup is in flight per handle: a second hadfl_backup_begin first
+ * waits for the previous one.  hadfl_backup_wait without a backup in flight returns HADFL_OK. */
+int hadfl_backup_begin(hadfl_handle *h, int32_t device_id, float *dst, int64_t count);
+int hadfl_backup_wait(hadfl_handle *h);
+
 /* Versions v_i ("actual parameter version of device i", Section "Runtime information prediction")
  * and per-device step counters (the index into each device's gradient stream).  N entries each;
  * either pointer may be NULL.  Restoring w, m, versions and step counters resumes a run exactly. */

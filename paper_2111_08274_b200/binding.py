@@ -74,6 +74,8 @@ SIGNATURES = {
     "hadfl_read_momentum": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_write_params": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_write_momentum": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
+    "hadfl_backup_begin": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
+    "hadfl_backup_wait": (C.c_int, [_H]),
     "hadfl_get_versions": (C.c_int, [_H, _u32p, _u64p]),
     "hadfl_set_versions": (C.c_int, [_H, _u32p, _u64p]),
     "hadfl_set_available": (C.c_int, [_H, _u8p]),
@@ -279,6 +281,16 @@ class Hadfl:
 
     def read_momentum(self, device_id, count=None, out=None):
         return self._read(self._lib.hadfl_read_momentum, "hadfl_read_momentum", device_id, count, out)
+
+    def backup_begin(self, device_id, out, count=None):
+        """out: a host buffer of at least `count` floats that stays alive until backup_wait (a
+        pinned torch tensor or a numpy array)."""
+        count = self.n_params if count is None else int(count)
+        ptr = out.ctypes.data if isinstance(out, np.ndarray) else out.data_ptr()
+        self._check(self._lib.hadfl_backup_begin(self._h, device_id, ptr, count), "hadfl_backup_begin")
+
+    def backup_wait(self):
+        self._check(self._lib.hadfl_backup_wait(self._h), "hadfl_backup_wait")
 
     def write_params(self, device_id, values):
         v = _arr(values, np.float32)

@@ -38,6 +38,14 @@ struct hadfl_handle {
   double *d_round_partials = nullptr;
   unsigned int *d_round_ticket = nullptr;
   int round_grid = 0;
+  // model backup that overlaps with later rounds: staging row + copy stream
+  void *d_backup = nullptr;
+  cudaStream_t backup_stream = nullptr;
+  cudaEvent_t backup_ready = nullptr, backup_done = nullptr;
+  bool backup_in_flight = false;
+  float *backup_dst = nullptr;
+  int64_t backup_count = 0;
+  std::vector<uint16_t> backup_bf16;  // host landing zone when w is stored as bf16
   int last_cuda_error = 0;
   uint64_t launches = 0;
 };
@@ -335,6 +343,7 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
 int hadfl_destroy(hadfl_handle *h) {
   if (!h) return HADFL_OK;
   DeviceGuard guard(h->device);
+  hadfl_backup_wait(h);
   cudaStreamSynchronize(h->stream);
   if (h->own_arena) {
     cudaFree(h->w);
@@ -345,6 +354,11 @@ int hadfl_destroy(hadfl_handle *h) {
   cudaFree(h->d_stats);
   cudaFree(h->d_round_partials);
   cudaFree(h->d_round_ticket);
+  if (h->backup_stream) cudaStreamSynchronize(h->backup_stream);
+  cudaFree(h->d_backup);
+  if (h->backup_ready) cudaEventDestroy(h->backup_ready);
+  if (h->backup_done) cudaEventDestroy(h->backup_done);
+  if (h->backup_stream) cudaStreamDestroy(h->backup_stream);
   delete h;
   return HADFL_OK;
 }
@@ -637,6 +651,56 @@ int hadfl_write_params(hadfl_handle *h, int32_t id, const float *src, int64_t co
 }
 int hadfl_write_momentum(hadfl_handle *h, int32_t id, const float *src, int64_t count) {
   return write_row(h, id, src, count, true);
+}
+
+int hadfl_backup_wait(hadfl_handle *h) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (!h->backup_in_flight) return HADFL_OK;
+  DeviceGuard guard(h->device);
+  HADFL_CUDA(h, cudaEventSynchronize(h->backup_done));
+  h->backup_in_flight = false;
+  if (h->cfg.dtype == HADFL_DTYPE_BF16) {
+    for (int64_t p = 0; p < h->backup_count; ++p) {
+      const uint32_t bits = (uint32_t)h->backup_bf16[(size_t)p] << 16;
+      memcpy(h->backup_dst + p, &bits, 4);
+    }
+  }
+  return HADFL_OK;
+}
+
+int hadfl_backup_begin(hadfl_handle *h, int32_t device_id, float *dst, int64_t count) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (!dst || device_id < 0 || device_id >= h->cfg.n_devices || count < 1 || count > h->cfg.n_params)
+    return HADFL_ERR_INVALID;
+  if (h->backup_in_flight) {  // one backup at a time: finish the previous one first
+    const int rc = hadfl_backup_wait(h);
+    if (rc != HADFL_OK) return rc;
+  }
+  DeviceGuard guard(h->device);
+  const size_t es = elem_size(h);
+  if (!h->backup_stream) {  // first use: staging row, copy stream, two events
+    HADFL_CUDA(h, cudaMalloc(&h->d_backup, (size_t)h->cfg.n_params * es));
+    HADFL_CUDA(h, cudaStreamCreateWithFlags(&h->backup_stream, cudaStreamNonBlocking));
+    HADFL_CUDA(h, cudaEventCreateWithFlags(&h->backup_ready, cudaEventDisableTiming));
+    HADFL_CUDA(h, cudaEventCreateWithFlags(&h->backup_done, cudaEventDisableTiming));
+  }
+  // Snapshot on the main stream (device to device, ~2 P bytes of HBM traffic), then the slow
+  // copy to the host on the copy stream, so that later rounds do not wait for PCIe.
+  const char *src = (const char *)h->w + (size_t)device_id * (size_t)h->stride * es;
+  HADFL_CUDA(h, cudaMemcpyAsync(h->d_backup, src, (size_t)count * es, cudaMemcpyDeviceToDevice, h->stream));
+  HADFL_CUDA(h, cudaEventRecord(h->backup_ready, h->stream));
+  HADFL_CUDA(h, cudaStreamWaitEvent(h->backup_stream, h->backup_ready, 0));
+  void *host = dst;
+  if (h->cfg.dtype == HADFL_DTYPE_BF16) {
+    h->backup_bf16.resize((size_t)count);
+    host = h->backup_bf16.data();
+  }
+  HADFL_CUDA(h, cudaMemcpyAsync(host, h->d_backup, (size_t)count * es, cudaMemcpyDeviceToHost, h->backup_stream));
+  HADFL_CUDA(h, cudaEventRecord(h->backup_done, h->backup_stream));
+  h->backup_in_flight = true;
+  h->backup_dst = dst;
+  h->backup_count = count;
+  return HADFL_OK;
 }
 
 int hadfl_get_versions(hadfl_handle *h, uint32_t *versions, uint64_t *step_counts) {

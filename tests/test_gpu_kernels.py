@@ -365,3 +365,28 @@ def test_state_errors():
     assert list(h.get_versions()[1]) == [2**56 - 3, 0]
     h.local_step([0, 1], [2, 1], 0.01)      # up to the limit is fine
     assert list(h.get_versions()[1]) == [2**56 - 1, 1]
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_overlapped_backup_is_a_snapshot(dtype):
+    """hadfl_backup_begin captures the row as it is at that point of the stream, even though later
+    rounds (enqueued before the copy has finished) rewrite it."""
+    wl = small(3, 3_000_003, dtype=dtype)
+    h = gpu(wl)
+    h.local_step([0, 1, 2], [1, 2, 1], 0.01)
+    want = h.read_params(1)
+    buf = torch.empty(wl.n_params, dtype=torch.float32).pin_memory()
+    h.backup_begin(1, buf)
+    for r in range(3):                      # keeps the GPU busy rewriting row 1 while the copy runs
+        h.round([0, 1, 2], [2, 3, 1], 0.01, r, 2, 11)
+    h.backup_wait()
+    assert np.array_equal(buf.numpy(), want)
+    assert not np.array_equal(h.read_params(1), want)
+    h.backup_wait()                          # nothing in flight: no-op
+    part = np.empty(1000, dtype=np.float32)
+    h.backup_begin(1, part, count=1000)      # pageable memory works too
+    h.backup_begin(2, buf)                   # a second begin first finishes the one in flight
+    h.backup_wait()
+    assert np.array_equal(part, h.read_params(1)[:1000]) and np.array_equal(buf.numpy(), h.read_params(2))
+    with pytest.raises(binding.HadflError):
+        h.backup_begin(3, buf)
