@@ -16,7 +16,7 @@ per-replica statistics - one hadfl_round call, one kernel launch.  Prints ONE JS
             backup) into pinned host memory.
   roofline  for the kernel of the timed region (the fused round): algorithmic bytes per launch /
             average launch time (CUDA events around each launch), against the measured copy
-            bandwidth of this machine's B200s.
+            bandwidth of the B200 (MEASURED_PEAKS.json).
   cpu_baseline  the CPU checker (single thread, as it stands) on a column sample of the same
             workload, scaled to the full vector.
 
@@ -314,7 +314,7 @@ def run_ours(args, wl):
                 "what": "hadfl_local_step + hadfl_select + hadfl_aggregate + hadfl_stats_enqueue"}
     alu_peak = SM_COUNT * LANES_PER_CLK_PER_SM * SM_MAX_GHZ / ALU_INSTR_PER_ELEM_STEP   # Gelem-step/s
     alu_achieved = kernels["round"]["gelem_steps_per_s"]
-    hbm_src = ("of measured (copy bandwidth of this pool's B200s)" if peak_kind == "measured"
+    hbm_src = ("of measured (copy bandwidth, MEASURED_PEAKS.json)" if peak_kind == "measured"
                else "of fallback (6650 GB/s)")
     # which floor is higher for this launch: bytes / HBM peak or element-steps / issue peak?
     t_hbm, t_alu = round_bytes / (peak * 1e9), N * P * mean_steps / (alu_peak * 1e9)
