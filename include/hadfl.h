@@ -185,7 +185,7 @@ int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *ou
  * HADFL_ERR_INVALID; a failing CUDA call returns HADFL_ERR_CUDA.
  *
  * The first call on each device looks up the device address of the scratch array (once per
- * device); make that first call outside any stream capture.  All calls on a device share the one
+ * device); make that first call outside any stream capture and from one thread only.  All calls on a device share the one
  * array, which still holds what the previous call left there: each call re-zeroes the ticket on
  * the stream before its kernel, and two calls whose kernels overlap on the GPU (different streams,
  * no ordering between them) race on the scratch and give wrong sums - order them.  The result
