@@ -382,7 +382,7 @@ def run_ours(args, wl):
 
     arena.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        times, what = time_oracle(wl, 1.0 / 4.0, 3)
+        times, what = time_oracle(wl, 1.0 / 2.0, 3)
         line["cpu_baseline"] = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": 1,
                                 "kind": "oracle", "sample": what}
     if rank == 0:
