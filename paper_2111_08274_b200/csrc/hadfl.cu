@@ -146,15 +146,8 @@ int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
   constexpr int E = StepPack<WT>::E;
   const int64_t packs = (h->cfg.n_params + E - 1) / E;
   const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
-  int64_t total_steps = 0;
-  for (int j = 0; j < a.n; ++j) total_steps += a.r[j].steps;
-  const bool bandwidth_bound = sizeof(WT) == 2 && total_steps <= 2 * (int64_t)a.n;
-  if (bandwidth_bound)
-    k_local_step<WT, NormalsFast, E, 4><<<blocks, kThreads, 0, h->stream>>>(
-        (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
-  else
-    k_local_step<WT, NormalsFast, E, 1><<<blocks, kThreads, 0, h->stream>>>(
-        (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
+  k_local_step<WT, NormalsFast, E><<<blocks, kThreads, 0, h->stream>>>(
+      (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
   return check_launch(h);
 }
 

@@ -93,7 +93,7 @@ __device__ __forceinline__ void st_pack(__nv_bfloat16 *row, int64_t p, const flo
   }
 }
 // A loaded pack as it came from memory.  Loads fill a RawPack and nothing else, so that a thread
-// can issue all the loads of a batch (or the prefetch of the next row) without an instruction that
+// can issue all the loads of a batch (or both loads of a row) without an instruction that
 // depends on the data in between; `unpack` widens to fp32 registers at the point of use.
 template <typename WT, int E>
 struct RawPack;
@@ -319,8 +319,8 @@ k_init(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_para
 // K1: batched local update (Eq. 3 / Algorithm 1) for a list of devices with per-device step
 // counts, one launch.  A thread owns a pack of E columns (E/4 Philox blocks) and visits the listed
 // rows one after the other: load w and m once, run that device's steps in registers (gradient
-// from the counter-based generator), store once.  The next row's loads are issued before the
-// current row's arithmetic.  The gradient noise grad_std * z is produced directly (the scale is
+// from the counter-based generator), store once; other resident warps cover the load latency.
+// The gradient noise grad_std * z is produced directly (the scale is
 // folded into the constants of the radius), which differs from rounding z first by about one
 // part in 10^7.
 //
@@ -419,18 +419,14 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
 }
 
 // Row addressing: the host passes each row's byte offset, the thread adds the byte offset of its
-// pack once, so a row access costs one 64-bit add.  The row loop is unrolled by two with the two
-// register sets (current row / prefetched row) swapping roles, so nothing is copied.
+// pack once, so a row access costs one 64-bit add.
 template <typename WT>
 __device__ __forceinline__ WT *at_row(char *pack_in_row0, int64_t row_off) {
   return reinterpret_cast<WT *>(pack_in_row0 + row_off);
 }
 
-// MINB: resident blocks per SM the register allocation must allow.  With bf16 storage and few
-// steps per device the launch is bandwidth-bound and gains from a fourth resident block (64
-// registers); with many steps the unconstrained allocation is faster.  The host picks.
-template <typename WT, typename Gen, int E, int MINB>
-__global__ void __launch_bounds__(kThreads, MINB)
+template <typename WT, typename Gen, int E>
+__global__ void __launch_bounds__(kThreads)
 k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalStepArgs a,
              PhiloxKeys keys, StepConsts k) {
   const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -461,17 +457,14 @@ k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalS
       }
     }
   };
-  RawPack<WT, E> w0, w1;
-  RawPack<float, E> m0, m1;
-  load(0, w0, m0);
-  int j = 0;
-  for (; j + 1 < a.n; j += 2) {
-    load(j + 1, w1, m1);
-    visit(j, w0, m0);
-    if (j + 2 < a.n) load(j + 2, w0, m0);
-    visit(j + 1, w1, m1);
+  // No prefetch of the next row: the registers it would take cost a resident block, and four
+  // blocks per SM hide the row loads better than three blocks with a prefetch (measured).
+  RawPack<WT, E> rw;
+  RawPack<float, E> rm;
+  for (int j = 0; j < a.n; ++j) {
+    load(j, rw, rm);
+    visit(j, rw, rm);
   }
-  if (j < a.n) visit(j, w0, m0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -819,8 +812,8 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
         body(j, wv, rm.v);
       }
     };
-    // No prefetch of the next row here (unlike K1): the registers it would take cost a resident
-    // block, and three blocks per SM hide the row loads better than two blocks with a prefetch.
+    // No prefetch of the next row (as in K1): the registers it would take cost a resident block,
+    // and three blocks per SM hide the row loads better than two blocks with a prefetch.
     RawPack<WT, E> rw;
     RawPack<float, E> rm;
     zero_raw(rw);
