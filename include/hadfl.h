@@ -15,8 +15,9 @@
  *                        them (Eq. 5; Algorithm 1, "partial synchronization")
  *     hadfl_stats        per-replica squared norm and squared distance to a reference replica
  *                        (diagnostics; not in the paper)
- * and, when a model is wanted on the host (the coordinator's model backup, Section "Overall
- * Design" item 9), hadfl_read_params.
+ * or the single call hadfl_round, which runs that whole sequence in one kernel with identical
+ * results; and, when a model is wanted on the host (the coordinator's model backup, Section
+ * "Overall Design" item 9), hadfl_read_params or the overlapped hadfl_backup_begin / _wait.
  *
  * General rules
  *   - Every function returns an int status: HADFL_OK, HADFL_ERR_INVALID (bad argument, duplicate or
