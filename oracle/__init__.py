@@ -42,6 +42,10 @@ def _declare(l):
     l.oracle_select_bits.restype = C.c_uint64
     l.oracle_round_to_bf16.argtypes = [C.c_float]
     l.oracle_round_to_bf16.restype = C.c_float
+    l.oracle_round_to_bf16_stochastic.argtypes = [C.c_float, C.c_uint32]
+    l.oracle_round_to_bf16_stochastic.restype = C.c_float
+    l.oracle_rounding_words.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint32, _u32p]
+    l.oracle_rounding_words.restype = None
     l.oracle_third_quartile.argtypes = [_f64p, C.c_int]
     l.oracle_third_quartile.restype = C.c_double
     l.oracle_select_probs.argtypes = [_f64p, _u8p, C.c_int, _f64p]
@@ -51,7 +55,8 @@ def _declare(l):
     l.oracle_predict_version.argtypes = [_f64p, C.c_int, C.c_double, C.c_double]
     l.oracle_predict_version.restype = C.c_double
     l.oracle_sim_create.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_float, C.c_float, C.c_float,
-                                    C.c_float, C.c_uint64, C.c_double, C.c_int, _u32p, C.c_int64]
+                                    C.c_float, C.c_uint64, C.c_double, C.c_int, _u32p, C.c_int64,
+                                    C.c_int, C.c_int]
     l.oracle_sim_create.restype = C.c_void_p
     l.oracle_sim_destroy.argtypes = [C.c_void_p]
     l.oracle_sim_destroy.restype = None
@@ -148,6 +153,16 @@ def round_to_bf16(v):
     return float(lib().oracle_round_to_bf16(float(v)))
 
 
+def round_to_bf16_stochastic(v, r16):
+    return float(lib().oracle_round_to_bf16_stochastic(float(v), int(r16)))
+
+
+def rounding_words(seed, group, last_step, device):
+    out = np.empty(4, dtype=np.uint32)
+    lib().oracle_rounding_words(seed, group, last_step, device, _ptr(out, C.c_uint32))
+    return out
+
+
 # ---- selection / prediction ------------------------------------------------------------------
 def third_quartile(x):
     x = _f64(x)
@@ -188,15 +203,16 @@ class Sim:
 
     def __init__(self, n_devices, n_params, dtype=0, momentum=0.9, weight_decay=5e-4,
                  grad_std=1e-2, init_std=0.05, seed=0, version_scale=1.0, weight_mode=0,
-                 groups=None):
+                 groups=None, m_dtype=0, rounding=0):
         self.n_devices, self.n_params, self.dtype = n_devices, n_params, dtype
+        self.m_dtype, self.rounding = m_dtype, rounding
         if groups is not None:
             groups = np.ascontiguousarray(np.asarray(groups, dtype=np.uint32))
         self.groups = groups
         self._h = lib().oracle_sim_create(n_devices, n_params, dtype, momentum, weight_decay,
                                           grad_std, init_std, seed, version_scale, weight_mode,
                                           _ptr(groups, C.c_uint32),
-                                          0 if groups is None else len(groups))
+                                          0 if groups is None else len(groups), m_dtype, rounding)
         if not self._h:
             raise OracleError("oracle_sim_create rejected its arguments")
         self.n_cols = int(lib().oracle_sim_n_cols(self._h))

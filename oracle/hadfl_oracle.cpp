@@ -19,6 +19,11 @@
 //                               quartile of the versions; N_p devices are then drawn one after
 //                               the other without replacement; the draw order is the ring order.
 //   * version prediction      - Eq. 7 (Brown's double exponential smoothing).
+//   * reduced-precision state - not in the paper: parameters (and optionally momentum) stored as
+//                               bf16, rounded once per call either to nearest even or
+//                               stochastically (round up in magnitude with probability equal to
+//                               the discarded fraction), the random bits from the counter-based
+//                               generator below.
 //   * synthetic gradients     - not in the paper: a counter-based generator (Philox4x32-10,
 //                               Salmon et al., SC'11) feeding a Box-Muller transform stands in
 //                               for forward/backward; each side implements it from the
@@ -82,6 +87,7 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 const uint32_t kTagInit = 0x49000000u;
 const uint32_t kTagGrad = 0x47000000u;
 const uint32_t kTagSelect = 0x53000000u;
+const uint32_t kTagRound = 0x52000000u;
 
 // Four 32-bit words -> four standard normals (Box-Muller, two pairs).
 // u = (x + 0.5) * 2^-32 lies strictly inside (0,1), so the logarithm is finite.
@@ -153,6 +159,34 @@ float round_to_bf16(float v) {
   float out;
   std::memcpy(&out, &bits, 4);
   return out;
+}
+
+// bf16 storage, stochastic rounding: the 16 random bits r are added to the fp32 bit pattern below
+// the bf16 mantissa and the sum is truncated, so a finite value moves to its neighbour of larger
+// magnitude with probability (discarded 16 bits) / 2^16 and keeps its truncation otherwise; the
+// expectation is the value itself.  Infinities and NaNs take the nearest-even path.
+float round_to_bf16_stochastic(float v, uint32_t r16) {
+  uint32_t bits;
+  std::memcpy(&bits, &v, 4);
+  if ((bits & 0x7F800000u) == 0x7F800000u) return round_to_bf16(v);
+  bits += (r16 & 0xFFFFu);
+  bits &= 0xFFFF0000u;
+  float out;
+  std::memcpy(&out, &bits, 4);
+  return out;
+}
+
+// Random words for the stochastic rounding at the end of a local-update call: one generator block
+// per column group, indexed like the gradient block of the call's last step but with its own tag.
+// Element `lane` of the group uses word `lane`: low half for the parameter, high half for the
+// momentum.
+void rounding_words(uint64_t seed, uint32_t group, uint64_t last_step, uint32_t device,
+                    uint32_t x[4]) {
+  uint32_t key[2];
+  key_of(seed, key);
+  const uint32_t ctr[4] = {group, (uint32_t)last_step, device,
+                           kTagRound | (uint32_t)((last_step >> 32) & 0xFFFFFFu)};
+  philox4x32_10(ctr, key, x);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -264,7 +298,9 @@ int selection_draw(const double* x, const uint8_t* avail, int n, int64_t round, 
 struct Sim {
   int n_devices = 0;
   int64_t n_params = 0;
-  int dtype = 0;  // 0: fp32 storage, 1: bf16 storage of w (momentum stays fp32)
+  int dtype = 0;     // 0: fp32 storage of w, 1: bf16 storage of w
+  int m_dtype = 0;   // 0: fp32 storage of the momentum, 1: bf16 (only with bf16 w)
+  int rounding = 0;  // bf16 stores of the local update: 0 nearest even, 1 stochastic
   float momentum = 0.f, weight_decay = 0.f, grad_std = 0.f, init_std = 0.f;
   uint64_t seed = 0;
   double version_scale = 1.0;
@@ -353,6 +389,13 @@ uint64_t oracle_select_bits(uint64_t seed, int64_t round, uint32_t t) {
   return select_bits(seed, round, t);
 }
 float oracle_round_to_bf16(float v) { return round_to_bf16(v); }
+float oracle_round_to_bf16_stochastic(float v, uint32_t r16) {
+  return round_to_bf16_stochastic(v, r16);
+}
+void oracle_rounding_words(uint64_t seed, uint32_t group, uint64_t last_step, uint32_t device,
+                           uint32_t* x) {
+  rounding_words(seed, group, last_step, device, x);
+}
 
 // ---- selection without a simulation (Eq. 8) -------------------------------------------------
 double oracle_third_quartile(const double* x, int n) {
@@ -387,9 +430,13 @@ double oracle_predict_version(const double* v, int n_obs, double alpha, double m
 void* oracle_sim_create(int n_devices, int64_t n_params, int dtype, float momentum,
                         float weight_decay, float grad_std, float init_std, uint64_t seed,
                         double version_scale, int weight_mode, const uint32_t* groups,
-                        int64_t n_groups) {
+                        int64_t n_groups, int m_dtype, int rounding) {
   if (n_devices < 1 || n_params < 1 || (dtype != 0 && dtype != 1)) return nullptr;
+  if ((m_dtype != 0 && m_dtype != 1) || (rounding != 0 && rounding != 1)) return nullptr;
+  if (dtype == 0 && (m_dtype != 0 || rounding != 0)) return nullptr;  // bf16 options need bf16 w
   Sim* s = new Sim;
+  s->m_dtype = m_dtype;
+  s->rounding = rounding;
   s->n_devices = n_devices;
   s->n_params = n_params;
   s->dtype = dtype;
@@ -440,8 +487,9 @@ int64_t oracle_sim_n_cols(void* p) { return ((Sim*)p)->n_cols; }
 //   g  = grad_std * z + wd * w      (one rounding for the product grad_std*z, then one fma)
 //   m  = mu * m + g                 (one fma)
 //   w  = w - lr * m                 (one fma)
-// With bf16 storage w is widened on entry, kept in fp32 through the steps of this call and
-// rounded once at its end.
+// With bf16 storage a value is widened on entry, kept in fp32 through the steps of this call and
+// rounded once at its end (to nearest even, or stochastically with the words of rounding_words).
+// A device that runs no step in the call is not touched at all.
 int oracle_sim_local_step(void* p, const int32_t* ids, const int32_t* steps, int n, float lr) {
   Sim* s = (Sim*)p;
   if (!ids || !steps || !ids_valid(s, ids, n)) return 1;
@@ -464,8 +512,22 @@ int oracle_sim_local_step(void* p, const int32_t* ids, const int32_t* steps, int
           w[c] = std::fmaf(-lr, m[c], w[c]);
         }
       }
-      if (s->dtype == 1 && steps[j] > 0)
-        for (int lane = 0; lane < 4; ++lane) w[4 * gl + lane] = round_to_bf16(w[4 * gl + lane]);
+      if (s->dtype == 1 && steps[j] > 0) {
+        uint32_t x[4] = {0u, 0u, 0u, 0u};
+        if (s->rounding == 1)
+          rounding_words(s->seed, s->groups[gl], s->step_count[dev] + (uint64_t)steps[j] - 1,
+                         (uint32_t)dev, x);
+        for (int lane = 0; lane < 4; ++lane) {
+          const int64_t c = 4 * gl + lane;
+          if (s->rounding == 1) {
+            w[c] = round_to_bf16_stochastic(w[c], x[lane] & 0xFFFFu);
+            if (s->m_dtype == 1) m[c] = round_to_bf16_stochastic(m[c], x[lane] >> 16);
+          } else {
+            w[c] = round_to_bf16(w[c]);
+            if (s->m_dtype == 1) m[c] = round_to_bf16(m[c]);
+          }
+        }
+      }
     }
     s->step_count[dev] += (uint64_t)steps[j];
     s->version[dev] += (uint32_t)steps[j];
@@ -571,7 +633,8 @@ int oracle_sim_write(void* p, int id, int which, const float* src) {
     for (int lane = 0; lane < 4; ++lane) {
       const int64_t c = 4 * gl + lane;
       if (!s->live(gl, lane)) continue;
-      row[c] = (which == 0 && s->dtype == 1) ? round_to_bf16(src[c]) : src[c];
+      const bool narrow = which == 0 ? s->dtype == 1 : s->m_dtype == 1;
+      row[c] = narrow ? round_to_bf16(src[c]) : src[c];
     }
   return 0;
 }
