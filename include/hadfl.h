@@ -3,7 +3,8 @@
  *
  * The method is HADFL (Cao et al., "HADFL: Heterogeneity-aware Decentralized Federated Learning
  * Framework", arXiv 2111.08274).  N simulated heterogeneous devices each hold a flat parameter
- * vector w (fp32, or bf16 storage) and an fp32 momentum vector m.  All replicas live in one
+ * vector w (fp32, or bf16 storage) and a momentum vector m (fp32, or bf16 storage next to bf16
+ * parameters).  All replicas live in one
  * device-memory arena: row i of w is device i's model, at w_ptr + i * row_stride_elems elements.
  *
  * One training round is the call sequence
@@ -55,6 +56,17 @@ extern "C" {
 #define HADFL_DTYPE_FP32 0 /* w stored as fp32 */
 #define HADFL_DTYPE_BF16 1 /* w stored as bf16, all arithmetic in fp32, one rounding per call */
 
+/* How the local update rounds what it stores as bf16 (once per call and value).  Not in the paper,
+ * which trains in fp32: with nearest-even storage an update below half a bf16 spacing is lost
+ * every time, with stochastic storage it survives on average.  Stochastic: the 16 random bits r are
+ * added to the fp32 bit pattern and the low 16 bits dropped, so a finite value moves to its
+ * neighbour of larger magnitude with probability (dropped bits) / 2^16 (infinities and NaNs are
+ * rounded to nearest).  r comes from the Philox4x32-10 block with key = seed and counter
+ * (p / 4, s mod 2^32, i, 'R' << 24 | s >> 32), s the index of the LAST step the call runs on device
+ * i: lane p mod 4 of the block, low half for the parameter, high half for the momentum. */
+#define HADFL_ROUND_NEAREST 0
+#define HADFL_ROUND_STOCHASTIC 1
+
 #define HADFL_WEIGHTS_UNIFORM 0 /* a_j = 1/k: Eq. 5 with K read as the number of selected devices */
 #define HADFL_WEIGHTS_VERSION 1 /* extension, not in the paper: a_j proportional to f(v_j) of Eq. 8 */
 
@@ -73,12 +85,17 @@ typedef struct hadfl_config {
   int32_t weight_mode;      /* HADFL_WEIGHTS_* */
   void *w_ptr;              /* DEVICE pointer to the parameter arena, or NULL: the library
                                allocates it (and the momentum arena) and frees it at destroy */
-  void *m_ptr;              /* DEVICE pointer to the fp32 momentum arena; NULL iff w_ptr is NULL */
+  void *m_ptr;              /* DEVICE pointer to the momentum arena (fp32, or bf16 per m_dtype);
+                               NULL iff w_ptr is NULL */
   int64_t row_stride_elems; /* elements between rows; 0 = P rounded up to a multiple of 32.
                                Must be >= P and a multiple of 8.  Caller-owned arenas must be
                                16-byte aligned, hold N * row_stride_elems elements each and outlive
                                the handle. */
   void *cuda_stream;        /* cudaStream_t on which all work is enqueued (NULL = default stream) */
+  int32_t m_dtype;          /* HADFL_DTYPE_* of the momentum; bf16 only together with bf16 parameters */
+  int32_t rounding;         /* HADFL_ROUND_* of the local update's bf16 stores; stochastic only with
+                               bf16 parameters.  Aggregation and global synchronisation always round
+                               to nearest even. */
 } hadfl_config;
 
 /* Algorithm 1, step 1 ("synchronize the initial models"): creates the handle on the current CUDA
@@ -95,8 +112,10 @@ int hadfl_destroy(hadfl_handle *h);
  * runs steps[j] >= 0 SGD steps on its own replica, in ONE kernel launch for all listed devices:
  *     g = fma(wd, w, grad_std * z);  m = fma(mu, m, g);  w = fma(-lr, m, w)
  * (momentum and weight decay follow the PyTorch SGD convention; Eq. 3 is mu = wd = 0).  w and m
- * are read and written once per call whatever the step count.  Afterwards the version and the
- * step counter of each listed device have grown by its step count.
+ * are read and written once per call whatever the step count; values stored as bf16 are widened on
+ * entry, kept in fp32 through the steps and rounded once at the end (per config.rounding).  A device
+ * listed with 0 steps is not touched.  Afterwards the version and the step counter of each listed
+ * device have grown by its step count.
  * device_ids: n distinct ids in [0, N); 1 <= n <= N.  Asynchronous. */
 int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
                      float lr);
@@ -200,7 +219,8 @@ int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t
                         void *cuda_stream);
 
 /* Model backup (Section "Overall Design", item 9) and checkpointing.  `count` elements starting at
- * parameter 0 of device_id; bf16 storage is widened to / rounded from fp32 (nearest even).
+ * parameter 0 of device_id; bf16 storage (of parameters or momentum) is widened to / rounded from
+ * fp32 (nearest even).
  * Reads synchronise; writes are ordered on the stream and have consumed src on return. */
 int hadfl_read_params(hadfl_handle *h, int32_t device_id, float *dst, int64_t count);
 int hadfl_read_momentum(hadfl_handle *h, int32_t device_id, float *dst, int64_t count);

@@ -16,6 +16,7 @@ OK, ERR_INVALID, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, 1, 2, 3, 4
 MAX_DEVICES = 32
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 WEIGHTS_UNIFORM, WEIGHTS_VERSION = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 
 
 class hadfl_config(C.Structure):
@@ -34,6 +35,8 @@ class hadfl_config(C.Structure):
         ("m_ptr", C.c_void_p),
         ("row_stride_elems", C.c_int64),
         ("cuda_stream", C.c_void_p),
+        ("m_dtype", C.c_int32),
+        ("rounding", C.c_int32),
     ]
 
 
@@ -163,12 +166,13 @@ class Hadfl:
 
     def __init__(self, n_devices, n_params, dtype=DTYPE_FP32, momentum=0.9, weight_decay=5e-4,
                  grad_std=1e-3, init_std=0.05, seed=0, version_scale=1.0, weight_mode=0,
-                 w_ptr=None, m_ptr=None, row_stride_elems=0, stream=0):
+                 w_ptr=None, m_ptr=None, row_stride_elems=0, stream=0, m_dtype=DTYPE_FP32,
+                 rounding=ROUND_NEAREST):
         self._lib = lib()
         self.n_devices, self.n_params, self.dtype = int(n_devices), int(n_params), int(dtype)
         cfg = hadfl_config(n_devices, n_params, dtype, momentum, weight_decay, grad_std, init_std,
                            seed, version_scale, weight_mode, w_ptr, m_ptr, row_stride_elems,
-                           stream or None)
+                           stream or None, m_dtype, rounding)
         h = _H()
         rc = self._lib.hadfl_init(C.byref(cfg), C.byref(h))
         self._h = h if h.value else None
@@ -181,7 +185,8 @@ class Hadfl:
     def from_workload(cls, wl, **kw):
         return cls(wl.n_devices, wl.n_params, dtype=wl.dtype, momentum=wl.momentum,
                    weight_decay=wl.weight_decay, grad_std=wl.grad_std, init_std=wl.init_std,
-                   seed=wl.seed, version_scale=wl.version_scale, weight_mode=wl.weight_mode, **kw)
+                   seed=wl.seed, version_scale=wl.version_scale, weight_mode=wl.weight_mode,
+                   m_dtype=wl.m_dtype, rounding=wl.rounding, **kw)
 
     def _check(self, rc, what):
         if rc:

@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "kernels.cuh"
@@ -19,7 +20,7 @@ struct hadfl_handle {
   hadfl_config cfg;
   int64_t stride = 0;
   void *w = nullptr;
-  float *m = nullptr;
+  void *m = nullptr;
   bool own_arena = false;
   cudaStream_t stream = nullptr;
   int device = 0;
@@ -53,6 +54,28 @@ struct hadfl_handle {
 namespace {
 
 inline size_t elem_size(const hadfl_handle *h) { return h->cfg.dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
+inline size_t m_elem_size(const hadfl_handle *h) { return h->cfg.m_dtype == HADFL_DTYPE_BF16 ? 2 : 4; }
+
+// Calls f(parameter storage type, momentum storage type, rounding mode) for the handle's storage
+// configuration: fp32 / fp32, or bf16 parameters with fp32 or bf16 momentum, each rounded to
+// nearest even (0) or stochastically (1) at the end of a local-update call.
+template <typename T>
+struct TypeTag {
+  using type = T;
+};
+template <int V>
+using IntTag = std::integral_constant<int, V>;
+
+template <typename F>
+int for_storage(const hadfl_handle *h, F &&f) {
+  if (h->cfg.dtype == HADFL_DTYPE_FP32) return f(TypeTag<float>{}, TypeTag<float>{}, IntTag<0>{});
+  const bool stochastic = h->cfg.rounding == HADFL_ROUND_STOCHASTIC;
+  if (h->cfg.m_dtype == HADFL_DTYPE_BF16)
+    return stochastic ? f(TypeTag<__nv_bfloat16>{}, TypeTag<__nv_bfloat16>{}, IntTag<1>{})
+                      : f(TypeTag<__nv_bfloat16>{}, TypeTag<__nv_bfloat16>{}, IntTag<0>{});
+  return stochastic ? f(TypeTag<__nv_bfloat16>{}, TypeTag<float>{}, IntTag<1>{})
+                    : f(TypeTag<__nv_bfloat16>{}, TypeTag<float>{}, IntTag<0>{});
+}
 
 constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
 
@@ -79,7 +102,7 @@ RowStep row_step(const hadfl_handle *h, int dev, uint64_t base, int steps) {
   const uint64_t dp = (uint64_t)kPhiloxM1 * (uint32_t)dev;
   RowStep r;
   r.w_off = (int64_t)dev * h->stride * (int64_t)elem_size(h);
-  r.m_off = (int64_t)dev * h->stride * (int64_t)sizeof(float);
+  r.m_off = (int64_t)dev * h->stride * (int64_t)m_elem_size(h);
   r.row = dev;
   r.steps = steps;
   r.base_lo = (uint32_t)base;
@@ -132,42 +155,57 @@ int check_launch(hadfl_handle *h) {
   return HADFL_OK;
 }
 
-template <typename WT>
 int launch_init(hadfl_handle *h) {
-  const int64_t groups = h->stride / 4;
-  const unsigned blocks = (unsigned)((groups + kThreads - 1) / kThreads);
-  k_init<WT><<<blocks, kThreads, 0, h->stream>>>((WT *)h->w, h->m, h->stride, h->cfg.n_params,
-                                                 h->cfg.n_devices, h->keys, h->cfg.init_std);
-  return check_launch(h);
+  return for_storage(h, [&](auto wt, auto mt, auto) {
+    using WT = typename decltype(wt)::type;
+    using MT = typename decltype(mt)::type;
+    const int64_t groups = h->stride / 4;
+    const unsigned blocks = (unsigned)((groups + kThreads - 1) / kThreads);
+    k_init<WT, MT><<<blocks, kThreads, 0, h->stream>>>((WT *)h->w, (MT *)h->m, h->stride,
+                                                       h->cfg.n_params, h->cfg.n_devices, h->keys,
+                                                       h->cfg.init_std);
+    return check_launch(h);
+  });
 }
 
-template <typename WT>
 int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
-  constexpr int E = StepPack<WT>::E;
-  const int64_t packs = (h->cfg.n_params + E - 1) / E;
-  const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
-  k_local_step<WT, NormalsFast, E><<<blocks, kThreads, 0, h->stream>>>(
-      (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
-  return check_launch(h);
+  return for_storage(h, [&](auto wt, auto mt, auto rm) {
+    using WT = typename decltype(wt)::type;
+    using MT = typename decltype(mt)::type;
+    constexpr int E = StepPack<WT>::E;
+    const int64_t packs = (h->cfg.n_params + E - 1) / E;
+    const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
+    k_local_step<WT, MT, NormalsFast, E, decltype(rm)::value><<<blocks, kThreads, 0, h->stream>>>(
+        (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
+    return check_launch(h);
+  });
 }
 
-template <typename WT>
 int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
-  const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
-  k_round<WT, NormalsFast, StepPack<WT>::E><<<h->round_grid, kThreads, smem, h->stream>>>(
-      (WT *)h->w, h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-      h->d_round_ticket, h->d_stats);
-  return check_launch(h);
+  return for_storage(h, [&](auto wt, auto mt, auto rm) {
+    using WT = typename decltype(wt)::type;
+    using MT = typename decltype(mt)::type;
+    const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
+    k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value>
+        <<<h->round_grid, kThreads, smem, h->stream>>>((WT *)h->w, (MT *)h->m, h->cfg.n_params, a,
+                                                       h->keys, step_consts(h, lr),
+                                                       h->d_round_partials, h->d_round_ticket,
+                                                       h->d_stats);
+    return check_launch(h);
+  });
 }
 
-template <typename WT>
-int round_blocks_per_sm(int n_devices) {
-  int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-          &n, k_round<WT, NormalsFast, StepPack<WT>::E>, kThreads,
-          sizeof(float) * kThreads * (size_t)n_devices) != cudaSuccess || n < 1)
-    n = 1;
-  return n;
+int round_blocks_per_sm(const hadfl_handle *h) {
+  return for_storage(h, [&](auto wt, auto mt, auto rm) {
+    using WT = typename decltype(wt)::type;
+    using MT = typename decltype(mt)::type;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+            &n, k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value>, kThreads,
+            sizeof(float) * kThreads * (size_t)h->cfg.n_devices) != cudaSuccess || n < 1)
+      n = 1;
+    return n;
+  });
 }
 
 template <typename WT, int KR, int U>
@@ -210,15 +248,16 @@ int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool moment
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
     return HADFL_OK;
   }
-  if (momentum || h->cfg.dtype == HADFL_DTYPE_FP32) {
-    const float *src = (momentum ? h->m : (const float *)h->w) + (int64_t)id * h->stride;
+  const void *arena = momentum ? h->m : h->w;
+  if ((momentum ? m_elem_size(h) : elem_size(h)) == 4) {
+    const float *src = (const float *)arena + (int64_t)id * h->stride;
     HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost,
                                   h->stream));
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
     return HADFL_OK;
   }
   std::vector<uint16_t> tmp((size_t)count);
-  const uint16_t *src = (const uint16_t *)h->w + (int64_t)id * h->stride;
+  const uint16_t *src = (const uint16_t *)arena + (int64_t)id * h->stride;
   HADFL_CUDA(h, cudaMemcpyAsync(tmp.data(), src, 2 * (size_t)count, cudaMemcpyDeviceToHost, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
   for (int64_t p = 0; p < count; ++p) {
@@ -242,8 +281,9 @@ int write_row(hadfl_handle *h, int32_t id, const float *src, int64_t count, bool
   if (count == 0) return HADFL_OK;
   DeviceGuard guard(h->device);
   // The copy is ordered on the stream; waiting for it lets the caller reuse src at once.
-  if (momentum || h->cfg.dtype == HADFL_DTYPE_FP32) {
-    float *dst = (momentum ? h->m : (float *)h->w) + (int64_t)id * h->stride;
+  void *arena = momentum ? h->m : h->w;
+  if ((momentum ? m_elem_size(h) : elem_size(h)) == 4) {
+    float *dst = (float *)arena + (int64_t)id * h->stride;
     HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyHostToDevice,
                                   h->stream));
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
@@ -251,7 +291,7 @@ int write_row(hadfl_handle *h, int32_t id, const float *src, int64_t count, bool
   }
   std::vector<uint16_t> tmp((size_t)count);
   for (int64_t p = 0; p < count; ++p) tmp[(size_t)p] = bf16_bits_rn(src[p]);
-  uint16_t *dst = (uint16_t *)h->w + (int64_t)id * h->stride;
+  uint16_t *dst = (uint16_t *)arena + (int64_t)id * h->stride;
   HADFL_CUDA(h, cudaMemcpyAsync(dst, tmp.data(), 2 * (size_t)count, cudaMemcpyHostToDevice, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
   return HADFL_OK;
@@ -267,6 +307,12 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   if (cfg->n_devices < 1 || cfg->n_devices > HADFL_MAX_DEVICES) return HADFL_ERR_INVALID;
   if (cfg->n_params < 1 || cfg->n_params > ((int64_t)1 << 34) - 4) return HADFL_ERR_INVALID;
   if (cfg->dtype != HADFL_DTYPE_FP32 && cfg->dtype != HADFL_DTYPE_BF16) return HADFL_ERR_INVALID;
+  if (cfg->m_dtype != HADFL_DTYPE_FP32 && cfg->m_dtype != HADFL_DTYPE_BF16) return HADFL_ERR_INVALID;
+  if (cfg->rounding != HADFL_ROUND_NEAREST && cfg->rounding != HADFL_ROUND_STOCHASTIC)
+    return HADFL_ERR_INVALID;
+  // bf16 momentum and stochastic rounding are options of bf16 parameter storage
+  if (cfg->dtype == HADFL_DTYPE_FP32 && (cfg->m_dtype != HADFL_DTYPE_FP32 || cfg->rounding != HADFL_ROUND_NEAREST))
+    return HADFL_ERR_INVALID;
   if (cfg->weight_mode != HADFL_WEIGHTS_UNIFORM && cfg->weight_mode != HADFL_WEIGHTS_VERSION)
     return HADFL_ERR_INVALID;
   if ((cfg->w_ptr == nullptr) != (cfg->m_ptr == nullptr)) return HADFL_ERR_INVALID;
@@ -297,10 +343,10 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   if (!cfg->w_ptr) {
     h->own_arena = true;
     HADFL_CUDA(h, cudaMalloc(&h->w, elems * elem_size(h)));
-    HADFL_CUDA(h, cudaMalloc((void **)&h->m, elems * sizeof(float)));
+    HADFL_CUDA(h, cudaMalloc(&h->m, elems * m_elem_size(h)));
   } else {
     h->w = cfg->w_ptr;
-    h->m = (float *)cfg->m_ptr;
+    h->m = cfg->m_ptr;
   }
   // Statistics grid: one wave of resident blocks (8 blocks of 256 threads per SM), split evenly
   // over the rows; never more blocks per row than there are column chunks.
@@ -316,9 +362,7 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
   // Fused round kernel: one resident wave, never more blocks than there are packs to visit.
   {
-    const int per_sm = cfg->dtype == HADFL_DTYPE_BF16
-                           ? round_blocks_per_sm<__nv_bfloat16>(cfg->n_devices)
-                           : round_blocks_per_sm<float>(cfg->n_devices);
+    const int per_sm = round_blocks_per_sm(h);
     int64_t grid = (int64_t)h->sm_count * per_sm;
     const int64_t need = (packs + kThreads - 1) / kThreads;
     if (grid > need) grid = need;
@@ -330,7 +374,7 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
-  return cfg->dtype == HADFL_DTYPE_BF16 ? launch_init<__nv_bfloat16>(h) : launch_init<float>(h);
+  return launch_init(h);
 }
 
 int hadfl_destroy(hadfl_handle *h) {
@@ -389,8 +433,7 @@ int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *
       done[j] += take;
     }
     if (a.n > 0) {
-      const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_local_step<__nv_bfloat16>(h, a, lr)
-                                                      : launch_local_step<float>(h, a, lr);
+      const int rc = launch_local_step(h, a, lr);
       if (rc != HADFL_OK) return rc;
     }
     if (!more) break;
@@ -530,8 +573,7 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
     if (!(in_sel & (1u << i))) a.r[pos++] = row_step(h, i, h->step_count[i], row_steps[i]);
   {
     DeviceGuard guard(h->device);
-    const int rc = h->cfg.dtype == HADFL_DTYPE_BF16 ? launch_round<__nv_bfloat16>(h, a, lr)
-                                                    : launch_round<float>(h, a, lr);
+    const int rc = launch_round(h, a, lr);
     if (rc != HADFL_OK) return rc;
   }
   for (int i = 0; i < N; ++i) {

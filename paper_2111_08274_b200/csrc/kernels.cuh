@@ -294,9 +294,9 @@ __device__ __forceinline__ float4 normals_of_block(uint32_t c0, uint32_t c1, uin
 // (ragged group and row padding) are zeroed in both arenas.  One thread per column group of the
 // padded row.
 // ------------------------------------------------------------------------------------------
-template <typename WT>
+template <typename WT, typename MT>
 __global__ void __launch_bounds__(kThreads)
-k_init(WT *__restrict__ w, float *__restrict__ m, int64_t stride, int64_t n_params, int n_devices,
+k_init(WT *__restrict__ w, MT *__restrict__ m, int64_t stride, int64_t n_params, int n_devices,
        PhiloxKeys keys, float init_std) {
   const int64_t g = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (4 * g >= stride) return;
@@ -418,6 +418,42 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Reduced-precision state (a workload variant outside the paper, which trains in fp32): the one
+// rounding to bf16 at the end of a local-update call may be stochastic.  The 16 random bits are
+// added to the fp32 bit pattern below the bf16 mantissa and the sum is truncated: a finite value
+// moves to its neighbour of larger magnitude with probability (discarded bits) / 2^16, so the
+// expectation is the value itself.  Infinities and NaNs are rounded to nearest even.
+// The bits come from one Philox block per column group and call, counter
+// (group, index of the call's last step, device, 'R' << 24 | index >> 32): element `lane` of the
+// group takes the low half of word `lane` for its parameter and the high half for its momentum.
+// The result is exactly representable in bf16, so the conversion at the store changes nothing.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_stochastic(float v, uint32_t r16) {
+  const uint32_t bits = __float_as_uint(v);
+  if ((bits & 0x7F800000u) == 0x7F800000u) return __bfloat162float(__float2bfloat16_rn(v));
+  return __uint_as_float((bits + r16) & 0xFFFF0000u);
+}
+
+template <typename MT, int NB>
+__device__ __forceinline__ void round_stochastic(float (&w)[4 * NB], float (&m)[4 * NB], int64_t pack,
+                                                 const RowStep &rs, const PhiloxKeys &keys) {
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    uint32_t x0 = (uint32_t)(pack * NB + b);
+    uint32_t x1 = rs.base_lo + (uint32_t)rs.steps - 1u;
+    uint32_t x2 = (uint32_t)rs.row;
+    uint32_t x3 = rs.r1_c2 ^ keys.b[0] ^ (kTagGrad ^ kTagRound);  // tag | high bits of the step index
+    philox4x32_10(x0, x1, x2, x3, keys);
+    const uint32_t x[4] = {x0, x1, x2, x3};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      w[4 * b + i] = bf16_stochastic(w[4 * b + i], x[i] & 0xFFFFu);
+      if (sizeof(MT) == 2) m[4 * b + i] = bf16_stochastic(m[4 * b + i], x[i] >> 16);
+    }
+  }
+}
+
 // Row addressing: the host passes each row's byte offset, the thread adds the byte offset of its
 // pack once, so a row access costs one 64-bit add.
 template <typename WT>
@@ -425,42 +461,50 @@ __device__ __forceinline__ WT *at_row(char *pack_in_row0, int64_t row_off) {
   return reinterpret_cast<WT *>(pack_in_row0 + row_off);
 }
 
-template <typename WT, typename Gen, int E>
+// WT / MT: storage types of the parameters and of the momentum (bf16 momentum only with bf16
+// parameters); RM = 1: the bf16 stores of this call are rounded stochastically.
+template <typename WT, typename MT, typename Gen, int E, int RM>
 __global__ void __launch_bounds__(kThreads)
-k_local_step(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, LocalStepArgs a,
+k_local_step(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, LocalStepArgs a,
              PhiloxKeys keys, StepConsts k) {
   const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   const int live = live_of(n_params, p, E);
   if (live == 0) return;
   const GroupProducts<E / 4> gp(p);
   char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
-  char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(float));
+  char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
 
-  auto load = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+  auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
     ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-    ld_raw(at_row<float>(mp, a.r[j].m_off), live, rm);
+    ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
   };
   auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
     sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+    if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
     st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-    st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+    st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
   };
   // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
-  auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+  auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
     if (a.r[j].steps > 0) {
       if constexpr (sizeof(WT) == 4) {
         body(j, rw.v, rm.v);
-      } else {
+      } else if constexpr (sizeof(MT) == 4) {
         float wv[E];
         unpack(rw, wv);
         body(j, wv, rm.v);
+      } else {
+        float wv[E], mv[E];
+        unpack(rw, wv);
+        unpack(rm, mv);
+        body(j, wv, mv);
       }
     }
   };
   // No prefetch of the next row: the registers it would take cost a resident block, and four
   // blocks per SM hide the row loads better than three blocks with a prefetch (measured).
   RawPack<WT, E> rw;
-  RawPack<float, E> rm;
+  RawPack<MT, E> rm;
   for (int j = 0; j < a.n; ++j) {
     load(j, rw, rm);
     visit(j, rw, rm);
@@ -722,9 +766,9 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
   *slot += keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
 }
 
-template <typename WT, typename Gen, int E>
+template <typename WT, typename MT, typename Gen, int E, int RM>
 __global__ void __launch_bounds__(kThreads, 3)
-k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
+k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
         StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
   constexpr int kWarps = kThreads / 32;
@@ -745,15 +789,15 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
     const bool act = live > 0;
     const GroupProducts<E / 4> gp(p);
     char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
-    char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(float));
+    char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
     float acc[E];
 #pragma unroll
     for (int i = 0; i < E; ++i) acc[i] = 0.f;
 
-    auto load = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+    auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
       if (act) {
         ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-        if (a.r[j].steps > 0) ld_raw(at_row<float>(mp, a.r[j].m_off), live, rm);
+        if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
       }
     };
     // One row: its steps, then its part in the aggregation / synchronisation and in the sums.
@@ -761,7 +805,8 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
       const bool stepped = act && a.r[j].steps > 0;
       if (stepped) {
         sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-        st_pack_any(at_row<float>(mp, a.r[j].m_off), 0, live, mv);
+        if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
+        st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
 #pragma unroll
         for (int i = 0; i < E; ++i) wv[i] = i < live ? as_stored(wv[i], w) : 0.f;  // dead lanes stay 0
       }
@@ -803,19 +848,24 @@ k_round(WT *__restrict__ w, float *__restrict__ m, int64_t n_params, RoundArgs a
       }
     };
     // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
-    auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<float, E> &rm) {
+    auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
       if constexpr (sizeof(WT) == 4) {
         body(j, rw.v, rm.v);
-      } else {
+      } else if constexpr (sizeof(MT) == 4) {
         float wv[E];
         unpack(rw, wv);
         body(j, wv, rm.v);
+      } else {
+        float wv[E], mv[E];
+        unpack(rw, wv);
+        unpack(rm, mv);  // only used when the row runs steps (the momentum is loaded only then)
+        body(j, wv, mv);
       }
     };
     // No prefetch of the next row (as in K1): the registers it would take cost a resident block,
     // and three blocks per SM hide the row loads better than two blocks with a prefetch.
     RawPack<WT, E> rw;
-    RawPack<float, E> rm;
+    RawPack<MT, E> rm;
     zero_raw(rw);
     zero_raw(rm);
     for (int j = 0; j < a.n; ++j) {

@@ -23,6 +23,7 @@ constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 constexpr uint32_t kTagInit = 0x49000000u;    // 'I': initial model, counter (group, 0, 0, tag)
 constexpr uint32_t kTagGrad = 0x47000000u;    // 'G': gradients, counter (group, step, device, tag|step>>32)
 constexpr uint32_t kTagSelect = 0x53000000u;  // 'S': selection, counter (draw, 0, round, tag|round>>32)
+constexpr uint32_t kTagRound = 0x52000000u;   // 'R': stochastic rounding, counter (group, last step, device, tag|step>>32)
 
 struct PhiloxKeys {
   uint32_t a[10];  // round keys for the word-0 product

@@ -28,7 +28,8 @@ class Arena:
         self.stride = (wl.n_params + 31) // 32 * 32
         wdtype = torch.bfloat16 if wl.dtype == binding.DTYPE_BF16 else torch.float32
         self.w = torch.empty((wl.n_devices, self.stride), dtype=wdtype, device=self.device)
-        self.m = torch.empty((wl.n_devices, self.stride), dtype=torch.float32, device=self.device)
+        mdtype = torch.bfloat16 if wl.m_dtype == binding.DTYPE_BF16 else torch.float32
+        self.m = torch.empty((wl.n_devices, self.stride), dtype=mdtype, device=self.device)
         with torch.cuda.stream(self.stream):
             self.h = binding.Hadfl.from_workload(wl, w_ptr=self.w.data_ptr(), m_ptr=self.m.data_ptr(),
                                                  row_stride_elems=self.stride,

@@ -36,6 +36,8 @@ class Workload:
     version_scale: float = 1.0
     weight_mode: int = 0
     dtype: int = 0                      # 0 fp32 storage, 1 bf16 storage of w
+    m_dtype: int = 0                    # 0 fp32 storage of the momentum, 1 bf16 (with bf16 w only)
+    rounding: int = 0                   # bf16 stores of the local update: 0 nearest even, 1 stochastic
     seed: int = BASE_SEED
     sync_every: int = 0                 # >0: every that many rounds the aggregate is also sent to the unselected devices
 

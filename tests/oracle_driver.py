@@ -16,4 +16,4 @@ def make_sim(oracle, wl, groups=None):
     return oracle.Sim(wl.n_devices, wl.n_params, dtype=wl.dtype, momentum=wl.momentum,
                       weight_decay=wl.weight_decay, grad_std=wl.grad_std, init_std=wl.init_std,
                       seed=wl.seed, version_scale=wl.version_scale, weight_mode=wl.weight_mode,
-                      groups=groups)
+                      groups=groups, m_dtype=wl.m_dtype, rounding=wl.rounding)

@@ -1,5 +1,6 @@
 """The C-ABI library loads without a GPU, exports what include/hadfl.h declares, and its host-only
 planning functions (Eq. 8 selection, Eq. 7 prediction) agree with the oracle."""
+import ctypes as C
 import os
 import re
 
@@ -37,7 +38,9 @@ def test_config_struct_layout_matches_the_header():
     offs = {n: getattr(c, n).offset for n, _ in c._fields_}
     assert offs == {"n_devices": 0, "n_params": 8, "dtype": 16, "momentum": 20, "weight_decay": 24,
                     "grad_std": 28, "init_std": 32, "seed": 40, "version_scale": 48, "weight_mode": 56,
-                    "w_ptr": 64, "m_ptr": 72, "row_stride_elems": 80, "cuda_stream": 88}
+                    "w_ptr": 64, "m_ptr": 72, "row_stride_elems": 80, "cuda_stream": 88,
+                    "m_dtype": 96, "rounding": 100}
+    assert C.sizeof(c) == 104
 
 
 def test_host_selection_matches_oracle_bit_for_bit(lib, oracle):
