@@ -77,6 +77,7 @@ int for_storage(const hadfl_handle *h, F &&f) {
                     : f(TypeTag<__nv_bfloat16>{}, TypeTag<float>{}, IntTag<0>{});
 }
 
+constexpr int kRowPerBlockMaxSteps = 2;  // local update: one row per block up to this many steps
 constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
 
 // Columns per thread in the local-update and fused-round kernels: two Philox blocks (two 16-byte
@@ -175,7 +176,15 @@ int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
     constexpr int E = StepPack<WT>::E;
     const int64_t packs = (h->cfg.n_params + E - 1) / E;
     const unsigned blocks = (unsigned)((packs + kThreads - 1) / kThreads);
-    k_local_step<WT, MT, NormalsFast, E, decltype(rm)::value><<<blocks, kThreads, 0, h->stream>>>(
+    // One row per block when the launch is memory-bound throughout (fp32 storage, at most two steps
+    // per device); otherwise every block walks over all rows.  Measured at the ResNet-18 size, 8
+    // devices: 210 vs 226 us at 1 step, 215 vs 224 us at 2 steps; with 3 or more steps, mixed step
+    // counts or bf16 storage the row walk is as fast or faster.
+    int max_steps = 0;
+    for (int j = 0; j < a.n; ++j) max_steps = a.r[j].steps > max_steps ? a.r[j].steps : max_steps;
+    const bool row_per_block = sizeof(WT) == 4 && max_steps <= kRowPerBlockMaxSteps && a.n > 1;
+    const dim3 grid(blocks, row_per_block ? (unsigned)a.n : 1u);
+    k_local_step<WT, MT, NormalsFast, E, decltype(rm)::value><<<grid, kThreads, 0, h->stream>>>(
         (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr));
     return check_launch(h);
   });
@@ -428,7 +437,7 @@ int hadfl_local_step(hadfl_handle *h, const int32_t *device_ids, const int32_t *
         take = (int)room;
         more = true;
       }
-      if (take == 0 && done[j] > 0) continue;  // finished in an earlier launch
+      if (take == 0) continue;  // nothing to run (a device listed with 0 steps is not touched)
       a.r[a.n++] = row_step(h, dev, base, take);
       done[j] += take;
     }

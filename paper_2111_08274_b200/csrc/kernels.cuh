@@ -341,7 +341,7 @@ struct RowStep {
   uint32_t r1_c2;    // (tag | step_hi) ^ key_b[0]   (xor hi(M0 * group) -> word 2)
 };
 
-struct LocalStepArgs {
+struct LocalStepArgs {  // the host lists only devices that run at least one step
   int32_t n;
   RowStep r[kMaxDevices];
 };
@@ -486,26 +486,30 @@ k_local_step(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, LocalStep
   };
   // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
   auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
-    if (a.r[j].steps > 0) {
-      if constexpr (sizeof(WT) == 4) {
-        body(j, rw.v, rm.v);
-      } else if constexpr (sizeof(MT) == 4) {
-        float wv[E];
-        unpack(rw, wv);
-        body(j, wv, rm.v);
-      } else {
-        float wv[E], mv[E];
-        unpack(rw, wv);
-        unpack(rm, mv);
-        body(j, wv, mv);
-      }
+    if constexpr (sizeof(WT) == 4) {
+      body(j, rw.v, rm.v);
+    } else if constexpr (sizeof(MT) == 4) {
+      float wv[E];
+      unpack(rw, wv);
+      body(j, wv, rm.v);
+    } else {
+      float wv[E], mv[E];
+      unpack(rw, wv);
+      unpack(rm, mv);
+      body(j, wv, mv);
     }
   };
   // No prefetch of the next row: the registers it would take cost a resident block, and four
   // blocks per SM hide the row loads better than three blocks with a prefetch (measured).
+  // Grid: x = chunks of kThreads packs; y = 1: the block walks over all listed rows (every thread
+  // mixes light and heavy rows, so memory-bound and arithmetic-bound phases overlap), or
+  // y = number of rows: one row per block (eight times more, shorter blocks: no partial last
+  // wave, which is worth 5-7 % when every row is memory-bound).  The host chooses.
   RawPack<WT, E> rw;
   RawPack<MT, E> rm;
-  for (int j = 0; j < a.n; ++j) {
+  const int j_begin = gridDim.y > 1 ? (int)blockIdx.y : 0;
+  const int j_end = gridDim.y > 1 ? j_begin + 1 : a.n;
+  for (int j = j_begin; j < j_end; ++j) {
     load(j, rw, rm);
     visit(j, rw, rm);
   }

@@ -1,6 +1,6 @@
 """Bandwidth and rounds/s tables over the workloads (the metric is quoted against P).
 
-    python -m paper_2111_08274_b200.sweep [--what c5|configs|all] [--rounds 30] [--json out.json]
+    python -m paper_2111_08274_b200.sweep [--what c5|configs|variants|all] [--rounds 30] [--json out.json]
 
 For every case: warm-up rounds, then `--rounds` timed rounds with CUDA events around each launch.
 Prints markdown tables: per kernel the median launch time and the algorithmic GB/s (bytes that
@@ -22,6 +22,7 @@ def measure(wl, rounds, warmup=3):
     h = arena.h
     N, P, k = wl.n_devices, wl.n_params, wl.k
     ew = 2 if wl.dtype else 4
+    em = 2 if wl.m_dtype else 4
     r = 0
     for _ in range(warmup):
         arena.run_round(r)
@@ -57,13 +58,14 @@ def measure(wl, rounds, warmup=3):
     end.record()
     torch.cuda.synchronize()
     fused_ms = start.elapsed_time(end) / rounds
-    bytes_ = {"local_step": N * P * (2 * ew + 8), "aggregate": 2 * k * P * ew, "stats": N * P * ew}
+    bytes_ = {"local_step": N * P * 2 * (ew + em), "aggregate": 2 * k * P * ew, "stats": N * P * ew}
     arena.close()
-    res = {"workload": wl.name, "N": N, "P": P, "k": k, "storage": "bf16" if wl.dtype else "fp32",
+    storage = ("bf16" if wl.dtype else "fp32") + ("+bf16 m" if wl.m_dtype else "") + (" sr" if wl.rounding else "")
+    res = {"workload": wl.name, "N": N, "P": P, "k": k, "storage": storage,
            "mean_steps": float(np.mean([s.mean() for s in steps])),
-           "arena_mb": N * P * (ew + 4) / 1e6, "round_ms": total_ms, "rounds_per_s": 1e3 / total_ms,
+           "arena_mb": N * P * (ew + em) / 1e6, "round_ms": total_ms, "rounds_per_s": 1e3 / total_ms,
            "fused_round_ms": fused_ms, "fused_rounds_per_s": 1e3 / fused_ms,
-           "fused_gbs": N * P * (2 * ew + 8) / fused_ms / 1e6}
+           "fused_gbs": N * P * 2 * (ew + em) / fused_ms / 1e6}
     for n in names:
         res[n + "_us"] = ms[n] * 1e3
         res[n + "_gbs"] = bytes_[n] / ms[n] / 1e6
@@ -86,7 +88,7 @@ def table(rows, peak):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", default="all", choices=["c5", "configs", "all"])
+    ap.add_argument("--what", default="all", choices=["c5", "configs", "variants", "all"])
     ap.add_argument("--rounds", type=int, default=30)
     ap.add_argument("--peak", type=float, default=0.0, help="HBM GB/s to quote fractions of")
     ap.add_argument("--json", default="")
@@ -114,6 +116,14 @@ def main():
             for hetero in (False, True):
                 for lp in range(16, 28):
                     rows.append(measure(workloads.c5(lp, dtype=dtype, hetero=hetero), a.rounds))
+    if a.what in ("variants", "all"):
+        # reduced-precision state next to bf16 parameters: bf16 momentum, stochastic rounding
+        from dataclasses import replace
+        for hetero in (False, True):
+            for m_dtype, rounding in ((0, 0), (0, 1), (1, 0), (1, 1)):
+                base = workloads.c5(25, dtype=1, hetero=hetero)
+                name = base.name + ("_m16" if m_dtype else "") + ("_sr" if rounding else "")
+                rows.append(measure(replace(base, name=name, m_dtype=m_dtype, rounding=rounding), a.rounds))
     print(table(rows, peak))
     if a.json:
         with open(a.json, "w") as f:

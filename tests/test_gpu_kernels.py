@@ -111,7 +111,9 @@ def test_local_step_parity(oracle, P, dtype):
     h, sim = gpu(wl), make_sim(oracle, wl)
     rows = workloads.random_rows(n, P, seed=P)
     load_rows(h, sim, rows)
-    calls = [([0, 1, 2, 3, 4], [1, 2, 3, 4, 8]), ([3, 1], [5, 0]), ([4], [1]), ([2, 0, 4, 1, 3], [2, 2, 1, 7, 3])]
+    # step counts of at most 2 take the one-row-per-block launch (fp32), larger ones the row walk
+    calls = [([0, 1, 2, 3, 4], [1, 2, 3, 4, 8]), ([3, 1], [5, 0]), ([4], [1]), ([2, 0, 4, 1, 3], [2, 2, 1, 7, 3]),
+             ([4, 2, 0, 1, 3], [1, 2, 1, 2, 2]), ([1, 3, 0], [2, 0, 1]), ([2, 4], [0, 0])]
     for ids, steps in calls:
         h.local_step(ids, steps, 0.01)
         sim.local_step(ids, steps, 0.01)
