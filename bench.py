@@ -55,7 +55,7 @@ ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to 
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum on a smaller case of the same kernel;
 # reads grow in proportion to the elements processed; writes are undercounted by whatever is still
 # dirty in the 126 MB L2 when the kernel ends).  None = not captured for the kernel as it stands.
-NCU_DRAM_BYTES_PER_ELEM = {"round": 14.25, "local_step": 14.29, "aggregate": 4.52, "stats": 4.12}
+NCU_DRAM_BYTES_PER_ELEM = {"round": 14.26, "local_step": 14.29, "aggregate": 4.58, "stats": 4.11}
 
 
 def measured_peak():
