@@ -10,7 +10,8 @@ per-replica statistics - one hadfl_round call, one kernel launch.  Prints ONE JS
             stream, barrier + synchronize on both sides, max over ranks.
   kernels / separate_calls   the same rounds as separate calls (hadfl_local_step, hadfl_select,
             hadfl_aggregate, hadfl_stats_enqueue) with CUDA events around every launch: the
-            bandwidth of each kernel on its own.
+            bandwidth of each kernel on its own; plus the local update at one step per device
+            (its memory-bound regime).
   e2e       the same rounds through the C ABI with HOST buffers: every round also reads the
             statistics (2N floats) and the aggregated model (P floats, the coordinator's model
             backup) into pinned host memory.
@@ -308,6 +309,22 @@ def run_ours(args, wl):
                       frac_key: gbs / peak, "frac_of_8TBs": gbs / 8000.0,
                       "share_of_separate_round": kern_ms[n] / sep_ms,
                       "traffic": None if per_elem is None else per_elem * units[n]}
+    # ---- the local update in its memory-bound regime: one step per device per call ---------------
+    Kb = max(3, min(K, 100))
+    ones = np.ones(N, dtype=np.int32)
+    ev1 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Kb)]
+    for _ in range(3):
+        h.local_step(ids, ones, wl.lr)
+    barrier()
+    for a, b in ev1:
+        a.record(); h.local_step(ids, ones, wl.lr); b.record()
+    barrier()
+    one_ms = float(np.mean([a.elapsed_time(b) for a, b in ev1]))
+    one_gbs = alg_bytes["local_step"] / (one_ms * 1e-3) / 1e9
+    kernels["local_step_1_step_per_device"] = {
+        "avg_ms": one_ms, "algorithmic_bytes": alg_bytes["local_step"], "achieved_gbs": one_gbs,
+        frac_key: one_gbs / peak, "frac_of_8TBs": one_gbs / 8000.0,
+        "traffic": NCU_DRAM_BYTES_PER_ELEM["local_step"] * N * P}
     kernels["local_step"]["mean_steps_per_device"] = sep_mean_steps
     kernels["local_step"]["gelem_steps_per_s"] = N * P * sep_mean_steps / (kern_ms["local_step"] * 1e-3) / 1e9
     separate = {"rounds_per_s": world * 1e3 / sep_ms, "ms_per_round": sep_ms, "rounds": Ks,

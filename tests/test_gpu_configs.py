@@ -51,14 +51,14 @@ def compare_sample(arena, sim, groups, what):
     return worst
 
 
-def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=()):
+def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=(), fused=False):
     arena = runtime.Arena(wl)
     sim = make_sim(oracle, wl, groups)
     full = groups is None
     g = np.arange((wl.n_params + 3) // 4, dtype=np.uint32) if full else groups
     worst = 0.0
     for r in range(wl.rounds):
-        sel = arena.run_round(r)
+        sel = arena.run_round_fused(r) if fused else arena.run_round(r)
         want_sel = oracle_round(sim, wl, r)
         assert np.array_equal(sel, want_sel), "round %d: selection %s != %s" % (r, sel, want_sel)
         v, s = arena.h.get_versions()
@@ -93,6 +93,20 @@ def test_c2_full_size_sampled_columns(oracle):
     wl = workloads.c2()
     groups = workloads.sample_groups(wl.n_params, 30_000, 1024, seed=2)
     run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24))
+
+
+def test_c2_full_size_fused_round_sampled_columns(oracle):
+    """The launch configuration the benchmark times: the whole round of the full-size workload in
+    one hadfl_round call per round."""
+    wl = workloads.c2()
+    groups = workloads.sample_groups(wl.n_params, 30_000, 1024, seed=22)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24), fused=True)
+
+
+def test_c3_full_size_fused_round_sampled_columns(oracle):
+    wl = workloads.c3()
+    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=33)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 10, 49), fused=True)
 
 
 def test_c2_shrunk_full_arena(oracle):
