@@ -789,8 +789,10 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
 
   for (int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x; p < n_packs_padded;
        p += (int64_t)gridDim.x * kThreads) {
+    // Lanes beyond the end (live = 0) take part in everything: their loads return zeros, their
+    // stores store nothing, and what they compute is zeroed before it is summed - so control flow
+    // stays uniform across the warp (the step loop's trip count is a launch parameter).
     const int live = live_of(n_params, p, E);
-    const bool act = live > 0;
     const GroupProducts<E / 4> gp(p);
     char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
     char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
@@ -799,20 +801,22 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
     for (int i = 0; i < E; ++i) acc[i] = 0.f;
 
     auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
-      if (act) {
-        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-        if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
-      }
+      ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+      if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
     };
     // One row: its steps, then its part in the aggregation / synchronisation and in the sums.
     auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
-      const bool stepped = act && a.r[j].steps > 0;
+      const bool stepped = a.r[j].steps > 0;
       if (stepped) {
         sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
         if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
         st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
 #pragma unroll
-        for (int i = 0; i < E; ++i) wv[i] = i < live ? as_stored(wv[i], w) : 0.f;  // dead lanes stay 0
+        for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
+        if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
+#pragma unroll
+          for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
+        }
       }
       if (j < a.k) {  // a selected device, visited in draw order: fold into the aggregate
         const float aj = a.a[j];
@@ -831,7 +835,7 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
             n2 = fmaf(acc[i], acc[i], n2);
           }
           // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
-          if (act && (a.k > 1 || a.r[0].steps > 0))
+          if (a.k > 1 || a.r[0].steps > 0)
             for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
           add_row_sums(s_acc, j, n2, 0.f, lane);  // one value for all selected devices
         }
@@ -840,7 +844,7 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
 #pragma unroll
           for (int i = 0; i < E; ++i) wv[i] = acc[i];
         }
-        if (act && (stepped || a.write_all)) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+        if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
         float n2 = 0.f, d2 = 0.f;
 #pragma unroll
         for (int i = 0; i < E; ++i) {
