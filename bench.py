@@ -49,6 +49,12 @@ FALLBACK_HBM_GBS = 6650.0
 # step loop = 2), i.e. 19 per parameter and step (ncu counts 78 in the kernel as it stands); an
 # SM issues 4 x 32 = 128 lane-instructions per clock.
 ALU_INSTR_PER_ELEM_STEP = 19.0
+# The same count weighted by issue cost: integer and conversion instructions run on 16-lane pipes
+# (64 results per clock and SM), so each holds the issue slot of its scheduler for two cycles.  Per
+# Philox block and step: 18 wide multiplies + 18 xors + 2 compares + 1 add + 4 conversions = 43
+# such instructions (86 slots) + 24 FP32 + 8 special-function + 1 branch = 119 slots, 29.75 per
+# parameter and step.  ncu measures 117 cycles per block and step in the local-update kernel.
+ALU_ISSUE_SLOTS_PER_ELEM_STEP = 29.75
 SM_COUNT, LANES_PER_CLK_PER_SM, SM_MAX_GHZ = 148, 128, 1.965
 ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to size its sample
 
@@ -331,6 +337,7 @@ def run_ours(args, wl):
                 "what": "hadfl_local_step + hadfl_select + hadfl_aggregate + hadfl_stats_enqueue"}
     alu_peak = SM_COUNT * LANES_PER_CLK_PER_SM * SM_MAX_GHZ / ALU_INSTR_PER_ELEM_STEP   # Gelem-step/s
     alu_achieved = kernels["round"]["gelem_steps_per_s"]
+    alu_peak_weighted = SM_COUNT * LANES_PER_CLK_PER_SM * SM_MAX_GHZ / ALU_ISSUE_SLOTS_PER_ELEM_STEP
     hbm_src = ("of measured (copy bandwidth, MEASURED_PEAKS.json)" if peak_kind == "measured"
                else "of fallback (6650 GB/s)")
     # which floor is higher for this launch: bytes / HBM peak or element-steps / issue peak?
@@ -348,6 +355,8 @@ def run_ours(args, wl):
                     "achieved": round_gbs, "peak": peak, "unit": "GB/s", "frac": round_gbs / peak,
                     "peak_source": hbm_src, "alu_achieved_gelem_steps": alu_achieved,
                     "alu_peak_gelem_steps": alu_peak, "alu_frac": alu_achieved / alu_peak}
+    roofline["alu_peak_half_rate_integer_gelem_steps"] = alu_peak_weighted
+    roofline["alu_frac_half_rate_integer"] = alu_achieved / alu_peak_weighted
     roofline["traffic"] = kernels["round"]["traffic"]
     roofline["note"] = ("algorithmic bytes = 16 per (device, parameter) whatever the step count; "
                         "mean steps per device here: %.2f; the bandwidth-bound kernels (local update "
