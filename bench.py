@@ -392,12 +392,22 @@ def run_ours(args, wl):
     torch.cuda.synchronize()
     blocking_s = max_over_ranks(time.perf_counter() - t0, world)
     r += Ke
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        arena.run_round_fused(r + i)
+        n2, d2 = h.stats_read()            # waits for the round: no launch runs ahead of the host
+    torch.cuda.synchronize()
+    stats_only_s = max_over_ranks(time.perf_counter() - t0, world)
+    r += Ke
     e2e = {"value": world * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": Ke,
            "what": "hadfl_round + hadfl_stats_read + hadfl_backup_begin/wait(selected[0]) into pinned "
                    "host memory, the model transfer overlapping the next round",
            "blocking_value": world * Ke / blocking_s,
-           "blocking_what": "the same with hadfl_read_params (waits for the transfer every round)"}
+           "blocking_what": "the same with hadfl_read_params (waits for the transfer every round)",
+           "stats_only_value": world * Ke / stats_only_s,
+           "stats_only_what": "hadfl_round + hadfl_stats_read only (2N floats back per round, no model copy)"}
 
     line = {"metric": METRIC, "value": world * K / (elapsed_ms * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": K, "warmup": warmup,
