@@ -771,7 +771,10 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
 }
 
 template <typename WT, typename MT, typename Gen, int E, int RM>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, sizeof(WT) == 2 ? 4 : 3)  // resident blocks per SM: with
+// bf16 parameters a row is 48 bytes per thread or less, and a fourth block (64 registers) buys more
+// bytes in flight than the tighter register budget costs (+10 % at one step per device); with fp32
+// parameters three blocks at 75 registers are faster (measured both ways)
 k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
         StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
@@ -871,7 +874,7 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
       }
     };
     // No prefetch of the next row (as in K1): the registers it would take cost a resident block,
-    // and three blocks per SM hide the row loads better than two blocks with a prefetch.
+    // and one more block per SM hides the row loads better than a prefetch.
     RawPack<WT, E> rw;
     RawPack<MT, E> rm;
     zero_raw(rw);
