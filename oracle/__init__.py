@@ -74,6 +74,8 @@ def _declare(l):
     l.oracle_sim_aggregate.restype = C.c_int
     l.oracle_sim_broadcast.argtypes = [C.c_void_p, C.c_int, _i32p, C.c_int]
     l.oracle_sim_broadcast.restype = C.c_int
+    l.oracle_sim_integrate.argtypes = [C.c_void_p, C.c_int, _i32p, C.c_int, C.c_float]
+    l.oracle_sim_integrate.restype = C.c_int
     l.oracle_sim_stats.argtypes = [C.c_void_p, C.c_int, _f64p, _f64p]
     l.oracle_sim_stats.restype = C.c_int
     l.oracle_sim_read.argtypes = [C.c_void_p, C.c_int, C.c_int, _f32p]
@@ -268,6 +270,11 @@ class Sim:
         dst = _i32(dst)
         self._check(lib().oracle_sim_broadcast(self._h, src, _ptr(dst, C.c_int32), len(dst)),
                     "broadcast")
+
+    def integrate(self, src, dst, beta):
+        dst = _i32(dst)
+        self._check(lib().oracle_sim_integrate(self._h, src, _ptr(dst, C.c_int32), len(dst), beta),
+                    "integrate")
 
     def stats(self, ref):
         n2 = np.empty(self.n_devices, dtype=np.float64)

@@ -19,6 +19,9 @@
 //                               quartile of the versions; N_p devices are then drawn one after
 //                               the other without replacement; the draw order is the ring order.
 //   * version prediction      - Eq. 7 (Brown's double exponential smoothing).
+//   * integration             - Section "Model aggregation and fault-tolerant": an unselected device
+//                               mixes the received model into its own (a reading offered beside the
+//                               overwrite of Algorithm 1; the paper gives no formula).
 //   * reduced-precision state - not in the paper: parameters (and optionally momentum) stored as
 //                               bf16, rounded once per call either to nearest even or
 //                               stochastically (round up in magnitude with probability equal to
@@ -595,6 +598,41 @@ int oracle_sim_broadcast(void* p, int src, const int32_t* dst, int n) {
   for (int j = 0; j < n; ++j) {
     std::memcpy(s->wrow(dst[j]), s->wrow(src), sizeof(float) * (size_t)s->n_cols);
     s->version[dst[j]] = s->version[src];
+  }
+  return 0;
+}
+
+// Global synchronisation read as a mix (Section "Model aggregation and fault-tolerant": the
+// unselected devices fold the received model into their own before the next local steps; the
+// paper gives no formula).  Reading offered beside the overwrite of Algorithm 1: a convex
+// combination with weight beta on the received model,
+//     w_dst = beta * w_src + (1 - beta) * w_dst,
+// evaluated as  t = (1 - beta) * w_dst  (1 - beta and the product rounded to float), then one fused
+// multiply-add  fma(beta, w_src, t).  beta = 1 reproduces the overwrite, beta = 0 leaves the
+// receiver as it is.  With bf16 storage the result is rounded to nearest even.  The receiver's
+// version becomes the larger of the two (it now carries both lineages), or the sender's when
+// beta = 1 (nothing of its own remains).
+int oracle_sim_integrate(void* p, int src, const int32_t* dst, int n, float beta) {
+  Sim* s = (Sim*)p;
+  if (src < 0 || src >= s->n_devices) return 1;
+  if (!(beta >= 0.0f && beta <= 1.0f)) return 1;
+  if (n == 0) return 0;
+  if (!dst || !ids_valid(s, dst, n)) return 1;
+  for (int j = 0; j < n; ++j)
+    if (dst[j] == src) return 1;
+  const float one_minus_beta = 1.0f - beta;
+  const float* from = s->wrow(src);
+  for (int j = 0; j < n; ++j) {
+    float* to = s->wrow(dst[j]);
+    for (int64_t c = 0; c < s->n_cols; ++c) {
+      const float t = one_minus_beta * to[c];
+      const float v = std::fmaf(beta, from[c], t);
+      to[c] = s->dtype == 1 ? round_to_bf16(v) : v;
+    }
+    if (beta == 1.0f)
+      s->version[dst[j]] = s->version[src];
+    else if (s->version[src] > s->version[dst[j]])
+      s->version[dst[j]] = s->version[src];
   }
   return 0;
 }
