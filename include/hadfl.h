@@ -152,6 +152,19 @@ int hadfl_aggregation_weights(hadfl_handle *h, const int32_t *selected, int32_t 
  * which also take its version.  One kernel: one read and n writes per element.  Asynchronous. */
 int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n);
 
+/* Global synchronisation read as a mix.  Section "Model aggregation and fault-tolerant" says that an
+ * unselected device folds the model it receives into its own parameters before its next local
+ * steps, without giving a formula; Algorithm 1 simply sends the model.  hadfl_broadcast is the
+ * second reading (overwrite), this call the first, as a convex combination with weight beta on the
+ * received model:
+ *     w[dst] = fma(beta, w[src], (1 - beta) * w[dst])      (1 - beta and the product rounded to fp32)
+ * for each of the n devices dst_ids (distinct, none equal to src, n may be 0); 0 <= beta <= 1.
+ * beta = 1 gives the overwrite, beta = 0 leaves the receivers as they are.  bf16 storage is rounded
+ * to nearest even.  Momentum is not touched.  A receiver's version becomes the larger of its own and
+ * the sender's (the sender's when beta = 1).  One kernel: 1 + n reads and n writes per element.
+ * Asynchronous. */
+int hadfl_integrate(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n, float beta);
+
 /* One whole round in ONE kernel: Algorithm 1's local steps of every listed device (Eq. 3), the
  * selection (Eq. 8), the partial aggregation with write-back (Eq. 5), optionally the global
  * synchronisation (Algorithm 1, "send w to devices whose Flag = 0": sync_all != 0 sends the

@@ -522,6 +522,42 @@ int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_
   return HADFL_OK;
 }
 
+int hadfl_integrate(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n, float beta) {
+  if (!h || src < 0 || src >= h->cfg.n_devices || n < 0) return HADFL_ERR_INVALID;
+  if (!(beta >= 0.0f && beta <= 1.0f)) return HADFL_ERR_INVALID;
+  if (n == 0) return HADFL_OK;
+  if (!distinct_ids(h, dst_ids, n)) return HADFL_ERR_INVALID;
+  for (int j = 0; j < n; ++j)
+    if (dst_ids[j] == src) return HADFL_ERR_INVALID;
+  MixArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = n;
+  a.src = src;
+  a.beta = beta;
+  a.one_minus_beta = 1.0f - beta;
+  for (int j = 0; j < n; ++j) a.dst[j] = dst_ids[j];
+  {
+    DeviceGuard guard(h->device);
+    constexpr int U = 2;
+    const int64_t pack_e = h->cfg.dtype == HADFL_DTYPE_BF16 ? 8 : 4;
+    const int64_t per_block = (int64_t)kThreads * U * pack_e;
+    const unsigned blocks = (unsigned)((h->cfg.n_params + per_block - 1) / per_block);
+    if (h->cfg.dtype == HADFL_DTYPE_BF16)
+      k_integrate<__nv_bfloat16, U><<<blocks, kThreads, 0, h->stream>>>((__nv_bfloat16 *)h->w, h->stride,
+                                                                     h->cfg.n_params, a);
+    else
+      k_integrate<float, U><<<blocks, kThreads, 0, h->stream>>>((float *)h->w, h->stride,
+                                                             h->cfg.n_params, a);
+    const int rc = check_launch(h);
+    if (rc != HADFL_OK) return rc;
+  }
+  for (int j = 0; j < n; ++j) {
+    uint32_t &v = h->version[dst_ids[j]];
+    if (beta == 1.0f || h->version[src] > v) v = h->version[src];
+  }
+  return HADFL_OK;
+}
+
 int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
                 int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
                 int32_t *out_selected) {

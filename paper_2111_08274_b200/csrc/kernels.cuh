@@ -615,6 +615,61 @@ k_combine(WT *__restrict__ w, int64_t stride, int64_t n_params, CombineArgs c) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Integration of a received model (Section "Model aggregation and fault-tolerant": an unselected
+// device folds the received parameters into its own; read here as a convex combination, beside the
+// overwrite that k_combine provides):
+//   w[dst_j] = fma(beta, w[src], (1 - beta) * w[dst_j])   for every receiver j,
+// the product rounded to fp32 before the fused multiply-add.  A thread owns U 16-byte packs; per
+// pack the sender's values are loaded once and the receivers' rows are loaded in batches of 8
+// before the batch's arithmetic and stores.  1 + n reads and n writes per element.
+// ------------------------------------------------------------------------------------------
+struct MixArgs {
+  int32_t n;    // receivers
+  int32_t src;  // sender
+  float beta, one_minus_beta;
+  int32_t dst[kMaxDevices];
+};
+
+template <typename WT, int U>
+__global__ void __launch_bounds__(kThreads)
+k_integrate(WT *__restrict__ w, int64_t stride, int64_t n_params, MixArgs a) {
+  constexpr int E = Pack16<WT>::E;
+  constexpr int B = 8;
+  const int64_t p0 = (int64_t)blockIdx.x * (kThreads * U) + threadIdx.x;
+  int live[U];
+  RawPack<WT, E> from[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int64_t p = p0 + (int64_t)u * kThreads;
+    live[u] = live_of(n_params, p, E);
+    if (live[u] > 0) ld_raw(w + (int64_t)a.src * stride + (int64_t)E * p, live[u], from[u]);
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    if (live[u] == 0) continue;
+    const int64_t p = p0 + (int64_t)u * kThreads;
+    float s[E];
+    unpack(from[u], s);
+    for (int base = 0; base < a.n; base += B) {
+      RawPack<WT, E> raw[B];
+#pragma unroll
+      for (int j = 0; j < B; ++j)
+        if (base + j < a.n) ld_raw(w + (int64_t)a.dst[base + j] * stride + (int64_t)E * p, live[u], raw[j]);
+#pragma unroll
+      for (int j = 0; j < B; ++j) {
+        if (base + j < a.n) {
+          float v[E];
+          unpack(raw[j], v);
+#pragma unroll
+          for (int i = 0; i < E; ++i) v[i] = fmaf(a.beta, s[i], __fmul_rn(a.one_minus_beta, v[i]));
+          st_pack_any(w + (int64_t)a.dst[base + j] * stride, p, live[u], v);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Deterministic reductions shared by the statistics kernel and the fused round kernel.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {

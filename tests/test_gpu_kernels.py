@@ -249,6 +249,45 @@ def test_broadcast(oracle, dtype):
     assert list(h.get_versions()[0]) == [9, 1, 9, 9, 4, 9]
 
 
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("P", [1, 5, 1023, 4099, 600_011])
+def test_integrate_bit_exact(oracle, P, dtype):
+    """The mix of a received model into the receivers' own: fixed fp32 arithmetic (one rounded
+    product, one fused multiply-add), so every stored bit equals the oracle's - for every number of
+    receivers, on ragged rows, with fp32 and bf16 storage."""
+    n = 32 if P <= 4099 else 6
+    wl = small(n, P, dtype=dtype)
+    h, sim = gpu(wl), make_sim(oracle, wl)
+    load_rows(h, sim, workloads.random_rows(n, P, seed=P + 3))
+    versions = np.arange(n, dtype=np.uint32)[::-1].copy()
+    rng = np.random.default_rng(P)
+    calls = [(0, [1], 0.5), (2, [0, 1, 3, 4, 5], 0.25), (1, [5, 0], 1.0), (3, [2], 0.0), (4, [], 0.7)]
+    if n == 32:
+        calls += [(7, [i for i in range(32) if i != 7], 0.1),
+                  (31, list(rng.permutation(31)[:17]), 0.9)]
+    for o in (h, sim):
+        o.set_versions(versions)
+        for src, dst, beta in calls:
+            o.integrate(src, dst, beta)
+    for i in range(n):
+        assert np.array_equal(h.read_params(i), sim.read_params(i)), i
+        assert not h.read_momentum(i).any()
+    assert np.array_equal(h.get_versions()[0], sim.get_versions()[0])
+
+
+def test_integrate_rejects_bad_arguments_and_leaves_the_arena_alone():
+    wl = small(4, 1000)
+    h = gpu(wl)
+    before = [h.read_params(i).copy() for i in range(4)]
+    for args in ((0, [0], 0.5), (0, [1, 1], 0.5), (4, [1], 0.5), (0, [7], 0.5), (0, [1], -0.1),
+                 (0, [1], 1.01), (0, [1], float("nan"))):
+        with pytest.raises(binding.HadflError) as e:
+            h.integrate(*args)
+        assert e.value.code == binding.ERR_INVALID
+    for i in range(4):
+        assert np.array_equal(h.read_params(i), before[i])
+
+
 # ---- K3 -----------------------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("n,P", [(1, 1), (4, 1003), (32, 4099), (7, 300_001), (16, 2_000_003)])
