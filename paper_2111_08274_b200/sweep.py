@@ -1,6 +1,6 @@
 """Bandwidth and rounds/s tables over the workloads (the metric is quoted against P).
 
-    python -m paper_2111_08274_b200.sweep [--what c5|configs|variants|all] [--rounds 30] [--json out.json]
+    python -m paper_2111_08274_b200.sweep [--what c5|configs|variants|sync|all] [--rounds 30] [--json out.json]
 
 For every case: warm-up rounds, then `--rounds` timed rounds with CUDA events around each launch.
 Prints markdown tables: per kernel the median launch time and the algorithmic GB/s (bytes that
@@ -72,6 +72,32 @@ def measure(wl, rounds, warmup=3):
     return res
 
 
+def measure_sync(wl, reps=30):
+    """Global synchronisation from device 0 to the N - k others: overwrite and beta-mix."""
+    arena = runtime.Arena(wl)
+    h = arena.h
+    ew = 2 if wl.dtype else 4
+    dst = np.arange(wl.k, wl.n_devices, dtype=np.int32)
+    out = {"workload": wl.name, "N": wl.n_devices, "P": wl.n_params, "receivers": len(dst),
+           "storage": "bf16" if wl.dtype else "fp32"}
+    for name, call, nbytes in (("broadcast", lambda: h.broadcast(0, dst), (1 + len(dst)) * wl.n_params * ew),
+                               ("integrate", lambda: h.integrate(0, dst, 0.5), (1 + 2 * len(dst)) * wl.n_params * ew)):
+        for _ in range(3):
+            call()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            call()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        out[name + "_us"] = ms * 1e3
+        out[name + "_gbs"] = nbytes / ms / 1e6
+    arena.close()
+    return out
+
+
 def table(rows, peak):
     out = ["| workload | N | P | k | storage | mean steps | arena MB | K1 µs | K1 GB/s (%% of %.0f) | K2 µs | K2 GB/s (%%) | K3 µs | K3 GB/s (%%) | round ms | rounds/s | fused round ms | fused rounds/s | fused GB/s (%%) |" % peak,
            "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
@@ -88,7 +114,7 @@ def table(rows, peak):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--what", default="all", choices=["c5", "configs", "variants", "all"])
+    ap.add_argument("--what", default="all", choices=["c5", "configs", "variants", "sync", "all"])
     ap.add_argument("--rounds", type=int, default=30)
     ap.add_argument("--peak", type=float, default=0.0, help="HBM GB/s to quote fractions of")
     ap.add_argument("--json", default="")
@@ -124,7 +150,21 @@ def main():
                 base = workloads.c5(25, dtype=1, hetero=hetero)
                 name = base.name + ("_m16" if m_dtype else "") + ("_sr" if rounding else "")
                 rows.append(measure(replace(base, name=name, m_dtype=m_dtype, rounding=rounding), a.rounds))
-    print(table(rows, peak))
+    sync_rows = []
+    if a.what in ("sync", "all"):
+        for wl in (workloads.c2(), workloads.c3(), workloads.c4(8), workloads.c5(25, dtype=1)):
+            sync_rows.append(measure_sync(wl))
+    if rows:
+        print(table(rows, peak))
+    if sync_rows:
+        print("\n| workload | N | P | receivers | storage | broadcast µs | GB/s (%% of %.0f) | integrate µs | GB/s (%%) |" % peak)
+        print("|---|---|---|---|---|---|---|---|---|")
+        for r in sync_rows:
+            print("| %s | %d | %d | %d | %s | %.1f | %.0f (%.0f) | %.1f | %.0f (%.0f) |" % (
+                r["workload"], r["N"], r["P"], r["receivers"], r["storage"], r["broadcast_us"],
+                r["broadcast_gbs"], 100 * r["broadcast_gbs"] / peak, r["integrate_us"],
+                r["integrate_gbs"], 100 * r["integrate_gbs"] / peak))
+        rows = rows + sync_rows
     if a.json:
         with open(a.json, "w") as f:
             json.dump(rows, f, indent=1)
