@@ -165,13 +165,19 @@ int hadfl_broadcast(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_
  * Asynchronous. */
 int hadfl_integrate(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_t n, float beta);
 
+/* Which reading hadfl_round's global synchronisation (sync_all != 0) takes: beta = 1 (the default)
+ * is the overwrite of hadfl_broadcast, 0 <= beta < 1 the mix of hadfl_integrate with that weight.
+ * Host only. */
+int hadfl_set_sync_beta(hadfl_handle *h, float beta);
+
 /* One whole round in ONE kernel: Algorithm 1's local steps of every listed device (Eq. 3), the
  * selection (Eq. 8), the partial aggregation with write-back (Eq. 5), optionally the global
  * synchronisation (Algorithm 1, "send w to devices whose Flag = 0": sync_all != 0 sends the
  * aggregate to every other device) and the statistics with the aggregate as reference.  It is
  * exactly the sequence
  *     hadfl_local_step(device_ids, steps, n, lr); hadfl_select(round, versions, seed, k);
- *     hadfl_aggregate(selected, k, versions); [hadfl_broadcast(selected[0], all others);]
+ *     hadfl_aggregate(selected, k, versions);
+ *     [hadfl_broadcast(selected[0], all others); or hadfl_integrate(..., beta), see hadfl_set_sync_beta]
  *     hadfl_stats_enqueue(selected[0])
  * - same parameters, momentum, versions and step counters, bit for bit - but each parameter and
  * momentum value is read and written once: the aggregate is formed in registers from the freshly

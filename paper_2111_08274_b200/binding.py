@@ -67,6 +67,7 @@ SIGNATURES = {
     "hadfl_aggregation_weights": (C.c_int, [_H, _i32p, C.c_int32, _f64p, _f32p]),
     "hadfl_broadcast": (C.c_int, [_H, C.c_int32, _i32p, C.c_int32]),
     "hadfl_integrate": (C.c_int, [_H, C.c_int32, _i32p, C.c_int32, C.c_float]),
+    "hadfl_set_sync_beta": (C.c_int, [_H, C.c_float]),
     "hadfl_round": (C.c_int, [_H, _i32p, _i32p, C.c_int32, C.c_float, C.c_int64, _f64p, C.c_uint64, C.c_int32,
                               C.c_int32, _i32p]),
     "hadfl_stats_enqueue": (C.c_int, [_H, C.c_int32]),
@@ -247,6 +248,9 @@ class Hadfl:
         dst = _arr(dst_ids, np.int32)
         self._check(self._lib.hadfl_integrate(self._h, src, _p(dst, C.c_int32), len(dst), beta),
                     "hadfl_integrate")
+
+    def set_sync_beta(self, beta):
+        self._check(self._lib.hadfl_set_sync_beta(self._h, beta), "hadfl_set_sync_beta")
 
     def round(self, device_ids, steps, lr, round_, k, seed, versions=None, sync_all=False):
         ids, st, v = _arr(device_ids, np.int32), _arr(steps, np.int32), _arr(versions, np.float64)

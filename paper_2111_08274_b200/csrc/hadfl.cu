@@ -47,6 +47,7 @@ struct hadfl_handle {
   float *backup_dst = nullptr;
   int64_t backup_count = 0;
   std::vector<uint16_t> backup_bf16;  // host landing zone when w is stored as bf16
+  float sync_beta = 1.0f;  // weight of the received model on global-synchronisation rounds of hadfl_round
   int last_cuda_error = 0;
   uint64_t launches = 0;
 };
@@ -558,6 +559,12 @@ int hadfl_integrate(hadfl_handle *h, int32_t src, const int32_t *dst_ids, int32_
   return HADFL_OK;
 }
 
+int hadfl_set_sync_beta(hadfl_handle *h, float beta) {
+  if (!h || !(beta >= 0.0f && beta <= 1.0f)) return HADFL_ERR_INVALID;
+  h->sync_beta = beta;
+  return HADFL_OK;
+}
+
 int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
                 int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
                 int32_t *out_selected) {
@@ -594,7 +601,8 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
       for (int j = 0; j < k; ++j) in_sel |= 1u << sel[j];
       for (int i = 0; i < N; ++i)
         if (!(in_sel & (1u << i))) others[n_others++] = i;
-      rc = hadfl_broadcast(h, sel[0], others, n_others);
+      rc = h->sync_beta == 1.0f ? hadfl_broadcast(h, sel[0], others, n_others)
+                                : hadfl_integrate(h, sel[0], others, n_others, h->sync_beta);
     }
     if (rc == HADFL_OK) rc = hadfl_stats_enqueue(h, sel[0]);
     if (rc != HADFL_OK) return rc;
@@ -606,7 +614,9 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
   memset(&a, 0, sizeof(a));
   a.n = N;
   a.k = k;
-  a.write_all = sync_all ? 1 : 0;
+  a.write_all = sync_all ? (h->sync_beta == 1.0f ? 1 : 2) : 0;
+  a.beta = h->sync_beta;
+  a.one_minus_beta = 1.0f - h->sync_beta;
   aggregation_weights(h->cfg.weight_mode, x, h->avail, N, sel, k, a.a);
   uint32_t in_sel = 0;
   int pos = 0;
@@ -629,7 +639,8 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
   for (int j = 0; j < k; ++j) vmax = h->version[sel[j]] > vmax ? h->version[sel[j]] : vmax;
   for (int j = 0; j < k; ++j) h->version[sel[j]] = vmax;
   if (sync_all)
-    for (int i = 0; i < N; ++i) h->version[i] = vmax;
+    for (int i = 0; i < N; ++i)
+      if (h->sync_beta == 1.0f || vmax > h->version[i]) h->version[i] = vmax;
   h->stats_valid = true;
   for (int j = 0; j < k; ++j) out_selected[j] = sel[j];
   return HADFL_OK;

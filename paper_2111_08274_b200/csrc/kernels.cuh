@@ -808,7 +808,9 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 struct RoundArgs {
   int32_t n;          // rows visited = all N devices: [0, k) selected in draw order, then the rest
   int32_t k;          // number of selected devices, 1 <= k <= n
-  int32_t write_all;  // 1: every device receives the aggregate (global synchronisation)
+  int32_t write_all;  // global synchronisation: 0 none, 1 every other device receives the aggregate
+                      // (overwrite), 2 every other device mixes it into its own model
+  float beta, one_minus_beta;  // weights of the mix (write_all = 2), as in k_integrate
   float a[kMaxDevices];  // aggregation weights of the selected devices
   RowStep r[kMaxDevices];
 };
@@ -898,9 +900,13 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
           add_row_sums(s_acc, j, n2, 0.f, lane);  // one value for all selected devices
         }
       } else {  // another device: keep its own model, or receive the aggregate
-        if (a.write_all) {
+        if (a.write_all == 1) {
 #pragma unroll
           for (int i = 0; i < E; ++i) wv[i] = acc[i];
+        } else if (a.write_all == 2) {
+#pragma unroll
+          for (int i = 0; i < E; ++i)
+            wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
         }
         if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
         float n2 = 0.f, d2 = 0.f;

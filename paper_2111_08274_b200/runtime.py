@@ -34,6 +34,8 @@ class Arena:
             self.h = binding.Hadfl.from_workload(wl, w_ptr=self.w.data_ptr(), m_ptr=self.m.data_ptr(),
                                                  row_stride_elems=self.stride,
                                                  stream=self.stream.cuda_stream)
+        if wl.sync_beta != 1.0:
+            self.h.set_sync_beta(wl.sync_beta)
         self.ids = wl.device_ids()
         self.select_seed = wl.select_seed()
 
@@ -59,7 +61,10 @@ class Arena:
         h.aggregate(sel)
         if wl.sync_every and (r + 1) % wl.sync_every == 0:
             others = np.setdiff1d(self.ids, sel).astype(np.int32)
-            h.broadcast(int(sel[0]), others)
+            if wl.sync_beta == 1.0:
+                h.broadcast(int(sel[0]), others)
+            else:
+                h.integrate(int(sel[0]), others, wl.sync_beta)
         if stats:
             h.stats_enqueue(int(sel[0]))
         return sel

@@ -40,6 +40,7 @@ class Workload:
     rounding: int = 0                   # bf16 stores of the local update: 0 nearest even, 1 stochastic
     seed: int = BASE_SEED
     sync_every: int = 0                 # >0: every that many rounds the aggregate is also sent to the unselected devices
+    sync_beta: float = 1.0              # weight of the received model on those rounds: 1 overwrite, <1 mix
 
     def steps_for_round(self, r: int) -> np.ndarray:
         """Step count of every device in round r (int32[n_devices])."""

@@ -8,7 +8,10 @@ def oracle_round(sim, wl, r):
     sim.aggregate(sel)
     if wl.sync_every and (r + 1) % wl.sync_every == 0:
         others = np.setdiff1d(wl.device_ids(), sel).astype(np.int32)
-        sim.broadcast(int(sel[0]), others)
+        if wl.sync_beta == 1.0:
+            sim.broadcast(int(sel[0]), others)
+        else:
+            sim.integrate(int(sel[0]), others, wl.sync_beta)
     return sel
 
 

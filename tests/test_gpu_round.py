@@ -63,6 +63,35 @@ def test_fused_round_equals_separate_calls(oracle, n, P, k, dtype):
     plain.close()
 
 
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("n,P,k,beta", [(6, 50_003, 2, 0.25), (8, 9_999, 4, 0.5), (5, 7, 1, 0.9), (4, 3_001, 4, 0.3)])
+def test_fused_round_with_mixed_global_synchronisation(oracle, n, P, k, beta, dtype):
+    """Global-synchronisation rounds that mix the aggregate into the unselected devices' own models
+    (hadfl_set_sync_beta) instead of overwriting them: the fused kernel against the separate calls
+    (hadfl_integrate) bit for bit, selections and versions against the oracle."""
+    wl = wl_of(n, P, k, dtype=dtype, sync_every=2, sync_beta=beta)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    sim = make_sim(oracle, wl)
+    for r in range(wl.rounds):
+        sf, sp, so = fused.run_round_fused(r), plain.run_round(r), oracle_round(sim, wl, r)
+        assert np.array_equal(sf, sp) and np.array_equal(sf, so), r
+        assert np.array_equal(fused.h.get_versions()[0], sim.get_versions()[0]), r
+        n2, d2 = fused.h.stats_read()
+        pn2, pd2 = plain.h.stats_read()
+        assert np.allclose(n2, pn2, rtol=2e-6) and np.allclose(d2, pd2, rtol=2e-6, atol=1e-30), r
+    assert_same_state(fused, plain, n)
+    for i in range(n):
+        got, want = fused.h.read_params(i), sim.read_params(i)
+        if dtype == 0:
+            assert_close_params(got, want, "w[%d]" % i)
+        else:
+            assert np.abs(got - want).max() <= 2 * bf16_ulp(np.abs(want).max()) and np.mean(got != want) < 0.02
+    with pytest.raises(binding.HadflError):
+        fused.h.set_sync_beta(1.5)
+    fused.close()
+    plain.close()
+
+
 def test_fused_round_subset_of_devices_zero_steps_mask_and_versions(oracle):
     """Only some devices step, one of them zero steps; an availability mask; caller-supplied versions."""
     wl = wl_of(6, 20_003, 2)
