@@ -109,6 +109,17 @@ def test_c3_full_size_fused_round_sampled_columns(oracle):
     run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 10, 49), fused=True)
 
 
+def test_c3_full_size_mixed_synchronisation_sampled_columns(oracle):
+    """Config 3 with the staleness-bounding synchronisation read as a mix (every 10th round the
+    unselected devices fold the aggregate into their own models with weight 1/2), through the
+    fused round and through the separate calls."""
+    from dataclasses import replace
+    wl = replace(workloads.c3(), rounds=30, sync_beta=0.5)
+    groups = workloads.sample_groups(wl.n_params, 4_000, 1024, seed=34)
+    run_and_compare(oracle, wl, groups, check_rounds=(9, 19), fused=True)
+    run_and_compare(oracle, wl, groups, check_rounds=(9, 19), fused=False)
+
+
 def test_c2_shrunk_full_arena(oracle):
     wl = workloads.shrink(workloads.c2(), 50_002, rounds=8)
     run_and_compare(oracle, wl, None, check_rounds=range(8), stats_rounds=range(8))
