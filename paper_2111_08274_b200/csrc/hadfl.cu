@@ -39,6 +39,7 @@ struct hadfl_handle {
   double *d_round_partials = nullptr;
   unsigned int *d_round_ticket = nullptr;
   int round_grid = 0;
+  int round_minb = 3;  // which instantiation of the fused round kernel: 3 or 4 resident blocks per SM
   // model backup that overlaps with later rounds: staging row + copy stream
   void *d_backup = nullptr;
   cudaStream_t backup_stream = nullptr;
@@ -196,24 +197,35 @@ int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
     using WT = typename decltype(wt)::type;
     using MT = typename decltype(mt)::type;
     const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
-    k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value>
-        <<<h->round_grid, kThreads, smem, h->stream>>>((WT *)h->w, (MT *)h->m, h->cfg.n_params, a,
-                                                       h->keys, step_consts(h, lr),
-                                                       h->d_round_partials, h->d_round_ticket,
-                                                       h->d_stats);
+    constexpr int E = StepPack<WT>::E;
+    constexpr int RM = decltype(rm)::value;
+    if (sizeof(WT) == 2 || h->round_minb == 4)
+      k_round<WT, MT, NormalsFast, E, RM, 4><<<h->round_grid, kThreads, smem, h->stream>>>(
+          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+          h->d_round_ticket, h->d_stats);
+    else if constexpr (sizeof(WT) == 4)
+      k_round<WT, MT, NormalsFast, E, RM, 3><<<h->round_grid, kThreads, smem, h->stream>>>(
+          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+          h->d_round_ticket, h->d_stats);
     return check_launch(h);
   });
 }
 
-int round_blocks_per_sm(const hadfl_handle *h) {
+// Resident blocks per SM of the fused round kernel compiled for `minb` blocks (bf16 parameters: 4 only).
+int round_blocks_per_sm(const hadfl_handle *h, int minb) {
   return for_storage(h, [&](auto wt, auto mt, auto rm) {
     using WT = typename decltype(wt)::type;
     using MT = typename decltype(mt)::type;
+    constexpr int E = StepPack<WT>::E;
+    constexpr int RM = decltype(rm)::value;
+    const size_t smem = sizeof(float) * kThreads * (size_t)h->cfg.n_devices;
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-            &n, k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value>, kThreads,
-            sizeof(float) * kThreads * (size_t)h->cfg.n_devices) != cudaSuccess || n < 1)
-      n = 1;
+    cudaError_t e;
+    if (sizeof(WT) == 2 || minb == 4)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_round<WT, MT, NormalsFast, E, RM, 4>, kThreads, smem);
+    else
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_round<float, float, NormalsFast, 8, 0, 3>, kThreads, smem);
+    if (e != cudaSuccess || n < 1) n = 1;
     return n;
   });
 }
@@ -371,10 +383,25 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_ticket, sizeof(unsigned int)));
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
   // Fused round kernel: one resident wave, never more blocks than there are packs to visit.
+  // A thread runs ceil(packs / resident threads) packs one after the other and the time follows that
+  // ceiling (a block left alone in a partly filled last pass runs barely faster), so with fp32
+  // parameters the 4-block instantiation is taken where its larger wave saves a whole pass:
+  // cost = passes x resident blocks per SM, 15 % extra for the 64-register code (measured 6-10 %).
   {
-    const int per_sm = round_blocks_per_sm(h);
+    const int64_t round_packs = (cfg->n_params + 7) / 8;
+    const int64_t need = (round_packs + kThreads - 1) / kThreads;
+    auto passes = [&](int per_sm) { return (need + (int64_t)h->sm_count * per_sm - 1) / ((int64_t)h->sm_count * per_sm); };
+    int per_sm = round_blocks_per_sm(h, cfg->dtype == HADFL_DTYPE_BF16 ? 4 : 3);
+    h->round_minb = cfg->dtype == HADFL_DTYPE_BF16 ? 4 : 3;
+    if (cfg->dtype == HADFL_DTYPE_FP32) {
+      const int per_sm4 = round_blocks_per_sm(h, 4);
+      if (per_sm4 > per_sm &&
+          1.15 * (double)(passes(per_sm4) * per_sm4) < (double)(passes(per_sm) * per_sm)) {
+        per_sm = per_sm4;
+        h->round_minb = 4;
+      }
+    }
     int64_t grid = (int64_t)h->sm_count * per_sm;
-    const int64_t need = (packs + kThreads - 1) / kThreads;
     if (grid > need) grid = need;
     h->round_grid = (int)grid;
   }

@@ -827,11 +827,13 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
   *slot += keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
 }
 
-template <typename WT, typename MT, typename Gen, int E, int RM>
-__global__ void __launch_bounds__(kThreads, sizeof(WT) == 2 ? 4 : 3)  // resident blocks per SM: with
-// bf16 parameters a row is 48 bytes per thread or less, and a fourth block (64 registers) buys more
-// bytes in flight than the tighter register budget costs (+10 % at one step per device); with fp32
-// parameters three blocks at 75 registers are faster (measured both ways)
+// MINB: resident blocks per SM the kernel is compiled for (3: 75 registers, 4: 64 registers with a
+// few bytes of spills).  With bf16 parameters a row is 48 bytes per thread or less and the fourth
+// block buys more bytes in flight than the tighter register budget costs (+10 % at one step per
+// device); with fp32 parameters three blocks are faster per element, and four are used only where
+// the larger wave saves a whole pass of the persistent loop (the host decides per handle).
+template <typename WT, typename MT, typename Gen, int E, int RM, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
         StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
