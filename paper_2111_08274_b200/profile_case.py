@@ -6,7 +6,8 @@
 The arena (N * P * 8 bytes for fp32) should exceed the 126 MB L2 so that DRAM counters mean
 something, and stay at a few hundred MB so that a multi-pass capture ends quickly.
 Launch order per repetition: local update once per entry of --steps (all devices that many
-steps), aggregation of k devices, statistics, broadcast to the other devices.  With --fused: one
+steps), aggregation of k devices, statistics, broadcast to the other devices, the same as a mix
+(beta = 1/2).  With --fused: one
 hadfl_round launch per entry of --steps instead.
 """
 import argparse
@@ -41,6 +42,7 @@ def main():
         ar.h.aggregate(sel)
         ar.h.stats_enqueue(int(sel[0]))
         ar.h.broadcast(int(sel[0]), ids[a.k:])
+        ar.h.integrate(int(sel[0]), ids[a.k:], 0.5)
     ar.h.synchronize()
     n2, d2 = ar.h.stats_read()
     print("ok: launches=%d norm2[0]=%.6g" % (ar.h.launch_count(), n2[0]))
