@@ -1,7 +1,8 @@
 // sm_100a kernels of the HADFL round: initial model (K0), batched heterogeneity-aware local
 // update (K1; Eq. 3 / Algorithm 1), fused weighted aggregation with write-back (K2; Eq. 5),
-// per-replica statistics (K3), and the fused round (K1 + K2 + global synchronisation + K3 in one
-// pass over the arena).
+// the mix of a received model into the receivers' own (Section "Model aggregation and
+// fault-tolerant"), per-replica statistics (K3), and the fused round (K1 + K2 + global
+// synchronisation + K3 in one pass over the arena).
 //
 // All of them stream rows of one [N][stride] arena.  A "column group" is four consecutive
 // parameters (one Philox block); a thread holds a "pack" of a row - 16 bytes of w in K2 / K3,
