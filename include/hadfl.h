@@ -191,6 +191,16 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
                 int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
                 int32_t *out_selected);
 
+/* A run of consecutive rounds enqueued by one call (the coordinator's loop of Algorithm 1 over the
+ * synchronisation rounds, for callers whose per-call overhead would otherwise bound small models):
+ * for i = 0 .. n_rounds-1, round r = first_round + i is exactly
+ *     hadfl_round(all N devices in id order, steps + i * N, N, lr, r, NULL, seed, k,
+ *                 sync_every > 0 && (r + 1) % sync_every == 0, out_selected + i * k)
+ * steps: n_rounds x N step counts; out_selected: n_rounds x k ids, or NULL.  Stops at the first
+ * round that fails and returns its status (earlier rounds stay enqueued).  Asynchronous. */
+int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const int32_t *steps, float lr,
+                 uint64_t seed, int32_t k, int32_t sync_every, int32_t *out_selected);
+
 /* Per-replica statistics (not in the paper; diagnostics of how far the replicas have drifted):
  * out_norm2[i] = sum_p w_i[p]^2, out_div2[i] = sum_p (w_i[p] - w_ref[p])^2, N floats each.
  * Deterministic: fixed grid, fixed summation order, fp32 within a chunk, fp64 above.

@@ -70,6 +70,7 @@ SIGNATURES = {
     "hadfl_set_sync_beta": (C.c_int, [_H, C.c_float]),
     "hadfl_round": (C.c_int, [_H, _i32p, _i32p, C.c_int32, C.c_float, C.c_int64, _f64p, C.c_uint64, C.c_int32,
                               C.c_int32, _i32p]),
+    "hadfl_rounds": (C.c_int, [_H, C.c_int64, C.c_int32, _i32p, C.c_float, C.c_uint64, C.c_int32, C.c_int32, _i32p]),
     "hadfl_stats_enqueue": (C.c_int, [_H, C.c_int32]),
     "hadfl_stats_read": (C.c_int, [_H, _f32p, _f32p]),
     "hadfl_stats": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
@@ -261,6 +262,16 @@ class Hadfl:
                                           round_, _p(v, C.c_double), seed, k, 1 if sync_all else 0,
                                           _p(out, C.c_int32)), "hadfl_round")
         return out[:k]
+
+    def rounds(self, first_round, steps, lr, k, seed, sync_every=0):
+        """steps: [n_rounds, N] step counts.  Returns the selected ids, [n_rounds, k]."""
+        st = np.ascontiguousarray(np.asarray(steps, dtype=np.int32))
+        if st.ndim != 2 or st.shape[1] != self.n_devices:
+            raise HadflError("hadfl_rounds", ERR_INVALID)
+        out = np.empty((st.shape[0], max(int(k), 1)), dtype=np.int32)
+        self._check(self._lib.hadfl_rounds(self._h, first_round, st.shape[0], _p(st, C.c_int32), lr, seed,
+                                           k, sync_every, _p(out, C.c_int32)), "hadfl_rounds")
+        return out[:, :k]
 
     def stats_enqueue(self, ref_device):
         self._check(self._lib.hadfl_stats_enqueue(self._h, ref_device), "hadfl_stats_enqueue")

@@ -673,6 +673,23 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
   return HADFL_OK;
 }
 
+int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const int32_t *steps, float lr,
+                 uint64_t seed, int32_t k, int32_t sync_every, int32_t *out_selected) {
+  if (!h || !steps || n_rounds < 0 || sync_every < 0) return HADFL_ERR_INVALID;
+  const int N = h->cfg.n_devices;
+  int32_t ids[kMaxDevices], sel[kMaxDevices];
+  for (int i = 0; i < N; ++i) ids[i] = i;
+  for (int32_t i = 0; i < n_rounds; ++i) {
+    const int64_t r = first_round + i;
+    const int32_t sync = sync_every > 0 && (r + 1) % sync_every == 0;
+    const int rc = hadfl_round(h, ids, steps + (int64_t)i * N, N, lr, r, nullptr, seed, k, sync, sel);
+    if (rc != HADFL_OK) return rc;
+    if (out_selected)
+      for (int j = 0; j < k; ++j) out_selected[(int64_t)i * k + j] = sel[j];
+  }
+  return HADFL_OK;
+}
+
 int hadfl_stats_enqueue(hadfl_handle *h, int32_t ref_device) {
   if (!h || ref_device < 0 || ref_device >= h->cfg.n_devices) return HADFL_ERR_INVALID;
   DeviceGuard guard(h->device);

@@ -51,6 +51,12 @@ class Arena:
         return self.h.round(self.ids, wl.steps_for_round(r), wl.lr, r, wl.k, self.select_seed,
                             sync_all=sync)
 
+    def run_rounds_fused(self, first_round, n_rounds):
+        """n_rounds consecutive rounds enqueued by ONE library call (hadfl_rounds)."""
+        wl = self.wl
+        steps = np.stack([wl.steps_for_round(first_round + i) for i in range(n_rounds)])
+        return self.h.rounds(first_round, steps, wl.lr, wl.k, self.select_seed, wl.sync_every)
+
     def run_round(self, r, stats=True):
         """One round of the hot path as separate calls: local steps of every device, selection,
         aggregation with write-back (plus, on the workload's global-synchronisation rounds, the

@@ -92,6 +92,26 @@ def test_fused_round_with_mixed_global_synchronisation(oracle, n, P, k, beta, dt
     plain.close()
 
 
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_a_run_of_rounds_in_one_call_equals_the_rounds_one_by_one(dtype):
+    from dataclasses import replace
+    wl = replace(workloads.shrink(workloads.c2(), 30_011, rounds=9), dtype=dtype, sync_every=4)
+    one, many = runtime.Arena(wl), runtime.Arena(wl)
+    want = np.stack([one.run_round_fused(r) for r in range(wl.rounds)])
+    got = np.concatenate([many.run_rounds_fused(0, 5), many.run_rounds_fused(5, 4)])
+    assert np.array_equal(got, want)
+    assert_same_state(one, many, wl.n_devices)
+    a, b = one.h.stats_read(), many.h.stats_read()
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert many.h.rounds(9, np.zeros((0, wl.n_devices), dtype=np.int32), wl.lr, wl.k, 1).shape == (0, wl.k)
+    with pytest.raises(binding.HadflError):
+        many.h.rounds(9, np.ones((2, wl.n_devices + 1), dtype=np.int32), wl.lr, wl.k, 1)
+    with pytest.raises(binding.HadflError):
+        many.h.rounds(9, np.ones((2, wl.n_devices), dtype=np.int32), wl.lr, wl.n_devices + 1, 1)
+    one.close()
+    many.close()
+
+
 def test_fused_round_subset_of_devices_zero_steps_mask_and_versions(oracle):
     """Only some devices step, one of them zero steps; an availability mask; caller-supplied versions."""
     wl = wl_of(6, 20_003, 2)
