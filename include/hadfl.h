@@ -232,8 +232,11 @@ int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *ou
  *
  * Limits: 1 <= n_devices <= HADFL_MAX_DEVICES and 1 <= n_params <= HADFL_NOALLOC_MAX_PARAMS;
  * anything larger returns HADFL_ERR_TOO_LARGE and enqueues nothing.  Other bad arguments (NULL or
- * misaligned pointers, stride < n_params or not a multiple of 8, ref_device out of range) return
- * HADFL_ERR_INVALID; a failing CUDA call returns HADFL_ERR_CUDA.
+ * misaligned pointers, a w or out_stats that is not device memory of the current device - checked
+ * with cudaPointerGetAttributes, so that a host pointer or another GPU's buffer is refused here
+ * instead of faulting in the kernel -, stride < n_params or not a multiple of 8, ref_device out of
+ * range) return HADFL_ERR_INVALID; a failing CUDA call returns HADFL_ERR_CUDA (an error left behind
+ * by earlier, unrelated CUDA work is cleared first and not reported).
  *
  * The first call on each device looks up the device address of the scratch array (once per
  * device); make that first call outside any stream capture and from one thread only.  All calls on a device share the one
@@ -248,6 +251,15 @@ int hadfl_stats(hadfl_handle *h, int32_t ref_device, float *out_norm2, float *ou
 int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t n_params,
                         int64_t row_stride_elems, int32_t ref_device, float *out_stats,
                         void *cuda_stream);
+
+/* The grid rule of the statistics kernel, as a pure host function (no GPU): blocks per row for a GPU
+ * with sm_count SMs - one wave of 8 blocks per SM split evenly over the n_devices rows, at most one
+ * block per 16 KB chunk of a row, and, when max_blocks > 0 (hadfl_stats_noalloc passes
+ * HADFL_NOALLOC_MAX_BLOCKS), at most max_blocks blocks in all.  Returns 0 for invalid arguments.
+ * With 148 SMs the cap of 2048 blocks is never reached (8 * 148 = 1184 resident blocks); it takes
+ * a GPU of more than 256 SMs. */
+int64_t hadfl_stats_grid_lanes(int32_t sm_count, int32_t n_devices, int64_t n_params, int32_t dtype,
+                               int64_t max_blocks);
 
 /* Model backup (Section "Overall Design", item 9) and checkpointing.  `count` elements starting at
  * parameter 0 of device_id; bf16 storage (of parameters or momentum) is widened to / rounded from
@@ -291,6 +303,10 @@ uint64_t hadfl_launch_count(const hadfl_handle *h);
 
 /* Row stride, in elements, of the handle's arenas. */
 int64_t hadfl_row_stride(const hadfl_handle *h);
+
+/* Number of thread blocks one hadfl_round launch of this handle uses (diagnostics; each block works
+ * on chunks of 2048 consecutive parameters of every device). */
+int32_t hadfl_round_grid(const hadfl_handle *h);
 
 /* ---- host-only functions (no handle, no GPU) ------------------------------------------------- */
 

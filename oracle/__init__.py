@@ -11,14 +11,27 @@ import numpy as np
 from . import build as _build
 
 _lib = None
+_lib_omp = None
 
 
-def lib():
-    global _lib
+def lib(openmp=False):
+    """The oracle library: the plain single-threaded build, or (openmp=True) the build of the same
+    source with -fopenmp that the all-cores CPU baseline times."""
+    global _lib, _lib_omp
+    if openmp:
+        if _lib_omp is None:
+            _lib_omp = C.CDLL(_build.build(openmp=True))
+            _declare(_lib_omp)
+        return _lib_omp
     if _lib is None:
         _lib = C.CDLL(_build.build())
         _declare(_lib)
     return _lib
+
+
+def threads(openmp=False):
+    """Threads the simulation loops of that build run on (1 for the plain build)."""
+    return int(lib(openmp).oracle_threads())
 
 
 _u32p = C.POINTER(C.c_uint32)
@@ -30,6 +43,8 @@ _f64p = C.POINTER(C.c_double)
 
 
 def _declare(l):
+    l.oracle_threads.argtypes = []
+    l.oracle_threads.restype = C.c_int
     l.oracle_philox4x32_10.argtypes = [_u32p, _u32p, _u32p]
     l.oracle_philox4x32_10.restype = None
     l.oracle_words_to_normals.argtypes = [_u32p, _f64p]
@@ -205,23 +220,24 @@ class Sim:
 
     def __init__(self, n_devices, n_params, dtype=0, momentum=0.9, weight_decay=5e-4,
                  grad_std=1e-2, init_std=0.05, seed=0, version_scale=1.0, weight_mode=0,
-                 groups=None, m_dtype=0, rounding=0):
+                 groups=None, m_dtype=0, rounding=0, openmp=False):
         self.n_devices, self.n_params, self.dtype = n_devices, n_params, dtype
         self.m_dtype, self.rounding = m_dtype, rounding
         if groups is not None:
             groups = np.ascontiguousarray(np.asarray(groups, dtype=np.uint32))
         self.groups = groups
-        self._h = lib().oracle_sim_create(n_devices, n_params, dtype, momentum, weight_decay,
+        self._lib = lib(openmp)
+        self._h = self._lib.oracle_sim_create(n_devices, n_params, dtype, momentum, weight_decay,
                                           grad_std, init_std, seed, version_scale, weight_mode,
                                           _ptr(groups, C.c_uint32),
                                           0 if groups is None else len(groups), m_dtype, rounding)
         if not self._h:
             raise OracleError("oracle_sim_create rejected its arguments")
-        self.n_cols = int(lib().oracle_sim_n_cols(self._h))
+        self.n_cols = int(self._lib.oracle_sim_n_cols(self._h))
 
     def close(self):
         if self._h:
-            lib().oracle_sim_destroy(self._h)
+            self._lib.oracle_sim_destroy(self._h)
             self._h = None
 
     def __del__(self):
@@ -236,56 +252,56 @@ class Sim:
 
     def local_step(self, ids, steps, lr):
         ids, steps = _i32(ids), _i32(steps)
-        self._check(lib().oracle_sim_local_step(self._h, _ptr(ids, C.c_int32), _ptr(steps, C.c_int32),
+        self._check(self._lib.oracle_sim_local_step(self._h, _ptr(ids, C.c_int32), _ptr(steps, C.c_int32),
                                                 len(ids), lr), "local_step")
 
     def select_probs(self, versions=None):
         v = _f64(versions)
         P = np.empty(self.n_devices, dtype=np.float64)
-        self._check(lib().oracle_sim_select_probs(self._h, _ptr(v, C.c_double), _ptr(P, C.c_double)),
+        self._check(self._lib.oracle_sim_select_probs(self._h, _ptr(v, C.c_double), _ptr(P, C.c_double)),
                     "select_probs")
         return P
 
     def select(self, round_, k, seed, versions=None):
         v = _f64(versions)
         out = np.empty(max(k, 1), dtype=np.int32)
-        self._check(lib().oracle_sim_select(self._h, round_, _ptr(v, C.c_double), seed, k,
+        self._check(self._lib.oracle_sim_select(self._h, round_, _ptr(v, C.c_double), seed, k,
                                             _ptr(out, C.c_int32)), "select")
         return out[:k]
 
     def aggregation_weights(self, selected, versions=None):
         sel, v = _i32(selected), _f64(versions)
         a = np.empty(len(sel), dtype=np.float32)
-        self._check(lib().oracle_sim_aggregation_weights(self._h, _ptr(sel, C.c_int32), len(sel),
+        self._check(self._lib.oracle_sim_aggregation_weights(self._h, _ptr(sel, C.c_int32), len(sel),
                                                          _ptr(v, C.c_double), _ptr(a, C.c_float)),
                     "aggregation_weights")
         return a
 
     def aggregate(self, selected, versions=None):
         sel, v = _i32(selected), _f64(versions)
-        self._check(lib().oracle_sim_aggregate(self._h, _ptr(sel, C.c_int32), len(sel),
+        self._check(self._lib.oracle_sim_aggregate(self._h, _ptr(sel, C.c_int32), len(sel),
                                                _ptr(v, C.c_double)), "aggregate")
 
     def broadcast(self, src, dst):
         dst = _i32(dst)
-        self._check(lib().oracle_sim_broadcast(self._h, src, _ptr(dst, C.c_int32), len(dst)),
+        self._check(self._lib.oracle_sim_broadcast(self._h, src, _ptr(dst, C.c_int32), len(dst)),
                     "broadcast")
 
     def integrate(self, src, dst, beta):
         dst = _i32(dst)
-        self._check(lib().oracle_sim_integrate(self._h, src, _ptr(dst, C.c_int32), len(dst), beta),
+        self._check(self._lib.oracle_sim_integrate(self._h, src, _ptr(dst, C.c_int32), len(dst), beta),
                     "integrate")
 
     def stats(self, ref):
         n2 = np.empty(self.n_devices, dtype=np.float64)
         d2 = np.empty(self.n_devices, dtype=np.float64)
-        self._check(lib().oracle_sim_stats(self._h, ref, _ptr(n2, C.c_double), _ptr(d2, C.c_double)),
+        self._check(self._lib.oracle_sim_stats(self._h, ref, _ptr(n2, C.c_double), _ptr(d2, C.c_double)),
                     "stats")
         return n2, d2
 
     def _read(self, i, which):
         out = np.empty(self.n_cols, dtype=np.float32)
-        self._check(lib().oracle_sim_read(self._h, i, which, _ptr(out, C.c_float)), "read")
+        self._check(self._lib.oracle_sim_read(self._h, i, which, _ptr(out, C.c_float)), "read")
         return out
 
     def read_cols(self, i):
@@ -308,7 +324,7 @@ class Sim:
         assert self.groups is None
         buf = np.zeros(self.n_cols, dtype=np.float32)
         buf[: self.n_params] = np.asarray(values, dtype=np.float32)
-        self._check(lib().oracle_sim_write(self._h, i, which, _ptr(buf, C.c_float)), "write")
+        self._check(self._lib.oracle_sim_write(self._h, i, which, _ptr(buf, C.c_float)), "write")
 
     def write_momentum(self, i, values):
         self.write_params(i, values, which=1)
@@ -316,19 +332,19 @@ class Sim:
     def write_cols(self, i, values, which=0):
         buf = np.ascontiguousarray(np.asarray(values, dtype=np.float32))
         assert buf.size == self.n_cols
-        self._check(lib().oracle_sim_write(self._h, i, which, _ptr(buf, C.c_float)), "write")
+        self._check(self._lib.oracle_sim_write(self._h, i, which, _ptr(buf, C.c_float)), "write")
 
     def get_versions(self):
         v = np.empty(self.n_devices, dtype=np.uint32)
         s = np.empty(self.n_devices, dtype=np.uint64)
-        lib().oracle_sim_get_versions(self._h, _ptr(v, C.c_uint32), _ptr(s, C.c_uint64))
+        self._lib.oracle_sim_get_versions(self._h, _ptr(v, C.c_uint32), _ptr(s, C.c_uint64))
         return v, s
 
     def set_versions(self, versions=None, step_counts=None):
         v = None if versions is None else np.ascontiguousarray(np.asarray(versions, dtype=np.uint32))
         s = None if step_counts is None else np.ascontiguousarray(np.asarray(step_counts, dtype=np.uint64))
-        lib().oracle_sim_set_versions(self._h, _ptr(v, C.c_uint32), _ptr(s, C.c_uint64))
+        self._lib.oracle_sim_set_versions(self._h, _ptr(v, C.c_uint32), _ptr(s, C.c_uint64))
 
     def set_available(self, mask=None):
         m = _u8(mask)
-        lib().oracle_sim_set_available(self._h, _ptr(m, C.c_uint8))
+        self._lib.oracle_sim_set_available(self._h, _ptr(m, C.c_uint8))

@@ -50,6 +50,18 @@
 #include <algorithm>
 #include <vector>
 
+// The oracle as it stands is single-threaded.  A second build with -fopenmp (oracle/build.py,
+// build(openmp=True)) runs the same loops split over column blocks on all host cores, only to time
+// an all-cores CPU baseline: every operation is elementwise in the column index, so the results
+// are identical bit for bit (tests/test_oracle_openmp.py); the statistics are split over replicas,
+// each summed sequentially as before.  Without -fopenmp the macro below is empty.
+#ifdef _OPENMP
+#include <omp.h>
+#define ORACLE_PARALLEL_FOR _Pragma("omp parallel for schedule(static)")
+#else
+#define ORACLE_PARALLEL_FOR
+#endif
+
 namespace {
 
 // ---------------------------------------------------------------------------------------
@@ -379,6 +391,15 @@ void aggregation_weights(const Sim* s, const int32_t* sel, int k, const double* 
 
 extern "C" {
 
+// Threads the loops above run on: 1 in the plain build.
+int oracle_threads() {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
 // ---- generator primitives (exposed for pins and for bit-level comparison) ----------------
 void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
   philox4x32_10(ctr, key, out);
@@ -502,6 +523,7 @@ int oracle_sim_local_step(void* p, const int32_t* ids, const int32_t* steps, int
     const int dev = ids[j];
     float* w = s->wrow(dev);
     float* m = s->mrow(dev);
+    ORACLE_PARALLEL_FOR
     for (int64_t gl = 0; gl < (int64_t)s->groups.size(); ++gl) {
       for (int e = 0; e < steps[j]; ++e) {
         float z[4];
@@ -574,6 +596,7 @@ int oracle_sim_aggregate(void* p, const int32_t* sel, int k, const double* versi
   if (!sel || !ids_valid(s, sel, k)) return 1;
   std::vector<float> a(k);
   aggregation_weights(s, sel, k, versions, a.data());
+  ORACLE_PARALLEL_FOR
   for (int64_t c = 0; c < s->n_cols; ++c) {
     float acc = a[0] * s->wrow(sel[0])[c];
     for (int j = 1; j < k; ++j) acc = std::fmaf(a[j], s->wrow(sel[j])[c], acc);
@@ -624,6 +647,7 @@ int oracle_sim_integrate(void* p, int src, const int32_t* dst, int n, float beta
   const float* from = s->wrow(src);
   for (int j = 0; j < n; ++j) {
     float* to = s->wrow(dst[j]);
+    ORACLE_PARALLEL_FOR
     for (int64_t c = 0; c < s->n_cols; ++c) {
       const float t = one_minus_beta * to[c];
       const float v = std::fmaf(beta, from[c], t);
@@ -641,6 +665,7 @@ int oracle_sim_integrate(void* p, int src, const int32_t* dst, int n, float beta
 int oracle_sim_stats(void* p, int ref, double* norm2, double* div2) {
   Sim* s = (Sim*)p;
   if (ref < 0 || ref >= s->n_devices) return 1;
+  ORACLE_PARALLEL_FOR
   for (int i = 0; i < s->n_devices; ++i) {
     double n2 = 0.0, d2 = 0.0;
     for (int64_t c = 0; c < s->n_cols; ++c) {

@@ -42,7 +42,8 @@ class hadfl_config(C.Structure):
 
 class HadflError(RuntimeError):
     def __init__(self, what, code, cuda_error=0):
-        names = {ERR_INVALID: "HADFL_ERR_INVALID", ERR_CUDA: "HADFL_ERR_CUDA", ERR_STATE: "HADFL_ERR_STATE"}
+        names = {ERR_INVALID: "HADFL_ERR_INVALID", ERR_CUDA: "HADFL_ERR_CUDA", ERR_STATE: "HADFL_ERR_STATE",
+                 ERR_TOO_LARGE: "HADFL_ERR_TOO_LARGE"}
         msg = "%s failed: %s" % (what, names.get(code, str(code)))
         if code == ERR_CUDA:
             msg += " (cudaError %d)" % cuda_error
@@ -76,6 +77,7 @@ SIGNATURES = {
     "hadfl_stats": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
     "hadfl_stats_noalloc": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
                                       C.c_void_p, C.c_void_p]),
+    "hadfl_stats_grid_lanes": (C.c_int64, [C.c_int32, C.c_int32, C.c_int64, C.c_int32, C.c_int64]),
     "hadfl_read_params": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_read_momentum": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
     "hadfl_write_params": (C.c_int, [_H, C.c_int32, C.c_void_p, C.c_int64]),
@@ -89,6 +91,7 @@ SIGNATURES = {
     "hadfl_last_cuda_error": (C.c_int, [_H]),
     "hadfl_launch_count": (C.c_uint64, [_H]),
     "hadfl_row_stride": (C.c_int64, [_H]),
+    "hadfl_round_grid": (C.c_int32, [_H]),
     "hadfl_selection_probs": (C.c_int, [_f64p, _u8p, C.c_int32, _f64p]),
     "hadfl_selection_draw": (C.c_int, [_f64p, _u8p, C.c_int32, C.c_int64, C.c_uint64, C.c_int32, _i32p]),
     "hadfl_predict_version": (C.c_int, [_f64p, C.c_int32, C.c_double, C.c_double, _f64p]),
@@ -156,6 +159,11 @@ def hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems, ref
     (see include/hadfl.h).  out_stats_ptr: 2N device floats, norm2 then div2.  Asynchronous."""
     return int(lib().hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems,
                                          ref_device, out_stats_ptr, stream or None))
+
+
+def hadfl_stats_grid_lanes(sm_count, n_devices, n_params, dtype=DTYPE_FP32, max_blocks=0):
+    """Blocks per row of a statistics launch on a GPU with sm_count SMs (host only)."""
+    return int(lib().hadfl_stats_grid_lanes(sm_count, n_devices, n_params, dtype, max_blocks))
 
 
 # ---- the handle --------------------------------------------------------------------------------
@@ -352,6 +360,9 @@ class Hadfl:
 
     def row_stride(self):
         return int(self._lib.hadfl_row_stride(self._h))
+
+    def round_grid(self):
+        return int(self._lib.hadfl_round_grid(self._h))
 
     def debug_philox(self, counters, key):
         c = _arr(counters, np.uint32).reshape(-1, 4)

@@ -36,10 +36,10 @@ struct hadfl_handle {
   int stats_lanes = 0;  // blocks per row of the statistics kernel
   bool stats_valid = false;
   // fused round kernel scratch
-  double *d_round_partials = nullptr;
-  unsigned int *d_round_ticket = nullptr;
+  double *d_round_partials = nullptr;        // [2 * kMaxDevices][round_grid]
+  double *d_round_group_partials = nullptr;  // [2 * kMaxDevices][groups of kFinishGroup blocks]
+  unsigned int *d_round_ticket = nullptr;    // [0]: the launch's ticket, [1 ...]: one per group
   int round_grid = 0;
-  int round_minb = 3;  // which instantiation of the fused round kernel: 3 or 4 resident blocks per SM
   // model backup that overlaps with later rounds: staging row + copy stream
   void *d_backup = nullptr;
   cudaStream_t backup_stream = nullptr;
@@ -81,6 +81,7 @@ int for_storage(const hadfl_handle *h, F &&f) {
 
 constexpr int kRowPerBlockMaxSteps = 2;  // local update: one row per block up to this many steps
 constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
+constexpr int64_t kRoundGridCap = 16384;  // most blocks of a fused-round launch (bounds its scratch: 8 MB)
 
 // Columns per thread in the local-update and fused-round kernels: two Philox blocks (two 16-byte
 // accesses of fp32 w, one of bf16 w).  Two independent generator chains per thread give the
@@ -89,6 +90,19 @@ template <typename WT>
 struct StepPack {
   static constexpr int E = 8;
 };
+
+// Blocks per row ("lanes") of a statistics launch: one wave of resident blocks (8 blocks of 256
+// threads per SM) split evenly over the rows, never more blocks per row than there are column
+// chunks, and - where the scratch is bounded - never more than max_blocks blocks in all.
+int64_t stats_lanes_for(int sm_count, int n_devices, int64_t n_params, int dtype, int64_t max_blocks) {
+  const int64_t pack_e = dtype == HADFL_DTYPE_BF16 ? 8 : 4;
+  const int64_t packs = (n_params + pack_e - 1) / pack_e;
+  const int64_t chunks = (packs + kThreads * kStatsU - 1) / (kThreads * kStatsU);
+  int64_t lanes = ((int64_t)sm_count * 8 + n_devices - 1) / n_devices;
+  if (lanes > chunks) lanes = chunks;
+  if (max_blocks > 0 && lanes * n_devices > max_blocks) lanes = max_blocks / n_devices;
+  return lanes < 1 ? 1 : lanes;
+}
 
 StepConsts step_consts(const hadfl_handle *h, float lr) {
   StepConsts k;
@@ -197,36 +211,10 @@ int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
     using WT = typename decltype(wt)::type;
     using MT = typename decltype(mt)::type;
     const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
-    constexpr int E = StepPack<WT>::E;
-    constexpr int RM = decltype(rm)::value;
-    if (sizeof(WT) == 2 || h->round_minb == 4)
-      k_round<WT, MT, NormalsFast, E, RM, 4><<<h->round_grid, kThreads, smem, h->stream>>>(
-          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-          h->d_round_ticket, h->d_stats);
-    else if constexpr (sizeof(WT) == 4)
-      k_round<WT, MT, NormalsFast, E, RM, 3><<<h->round_grid, kThreads, smem, h->stream>>>(
-          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-          h->d_round_ticket, h->d_stats);
+    k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value><<<h->round_grid, kThreads, smem, h->stream>>>(
+        (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+        h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
     return check_launch(h);
-  });
-}
-
-// Resident blocks per SM of the fused round kernel compiled for `minb` blocks (bf16 parameters: 4 only).
-int round_blocks_per_sm(const hadfl_handle *h, int minb) {
-  return for_storage(h, [&](auto wt, auto mt, auto rm) {
-    using WT = typename decltype(wt)::type;
-    using MT = typename decltype(mt)::type;
-    constexpr int E = StepPack<WT>::E;
-    constexpr int RM = decltype(rm)::value;
-    const size_t smem = sizeof(float) * kThreads * (size_t)h->cfg.n_devices;
-    int n = 0;
-    cudaError_t e;
-    if (sizeof(WT) == 2 || minb == 4)
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_round<WT, MT, NormalsFast, E, RM, 4>, kThreads, smem);
-    else
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_round<float, float, NormalsFast, 8, 0, 3>, kThreads, smem);
-    if (e != cudaSuccess || n < 1) n = 1;
-    return n;
   });
 }
 
@@ -370,45 +358,28 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
     h->w = cfg->w_ptr;
     h->m = cfg->m_ptr;
   }
-  // Statistics grid: one wave of resident blocks (8 blocks of 256 threads per SM), split evenly
-  // over the rows; never more blocks per row than there are column chunks.
-  const int64_t pack_e = cfg->dtype == HADFL_DTYPE_BF16 ? 8 : 4;
-  const int64_t packs = (cfg->n_params + pack_e - 1) / pack_e;
-  const int64_t chunks = (packs + kThreads * kStatsU - 1) / (kThreads * kStatsU);
-  int64_t lanes = ((int64_t)h->sm_count * 8 + cfg->n_devices - 1) / cfg->n_devices;
-  if (lanes > chunks) lanes = chunks;
+  const int64_t lanes = stats_lanes_for(h->sm_count, cfg->n_devices, cfg->n_params, cfg->dtype, 0);
   h->stats_lanes = (int)lanes;
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_partials,
                            sizeof(double) * 2 * (size_t)cfg->n_devices * (size_t)lanes));
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_ticket, sizeof(unsigned int)));
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_stats, sizeof(float) * 2 * kMaxDevices));
-  // Fused round kernel: one resident wave, never more blocks than there are packs to visit.
-  // A thread runs ceil(packs / resident threads) packs one after the other and the time follows that
-  // ceiling (a block left alone in a partly filled last pass runs barely faster), so with fp32
-  // parameters the 4-block instantiation is taken where its larger wave saves a whole pass:
-  // cost = passes x resident blocks per SM, 15 % extra for the 64-register code (measured 6-10 %).
+  // Fused round kernel: one block per chunk of kThreads packs (8 columns each) up to kRoundGridCap
+  // blocks, beyond which the blocks stride over the chunks.  Measured on the workloads' sizes, a grid
+  // of many short blocks beats one resident wave by 7-15 % with several steps per device and is
+  // equal at one step (caps of 592 / 1184 / 2368 / 4736 / 16384 blocks at the ResNet-18 size, 8
+  // devices, uniform 1..8 steps: 401 / 378 / 371 / 371 / 373 us).
   {
     const int64_t round_packs = (cfg->n_params + 7) / 8;
     const int64_t need = (round_packs + kThreads - 1) / kThreads;
-    auto passes = [&](int per_sm) { return (need + (int64_t)h->sm_count * per_sm - 1) / ((int64_t)h->sm_count * per_sm); };
-    int per_sm = round_blocks_per_sm(h, cfg->dtype == HADFL_DTYPE_BF16 ? 4 : 3);
-    h->round_minb = cfg->dtype == HADFL_DTYPE_BF16 ? 4 : 3;
-    if (cfg->dtype == HADFL_DTYPE_FP32) {
-      const int per_sm4 = round_blocks_per_sm(h, 4);
-      if (per_sm4 > per_sm &&
-          1.15 * (double)(passes(per_sm4) * per_sm4) < (double)(passes(per_sm) * per_sm)) {
-        per_sm = per_sm4;
-        h->round_minb = 4;
-      }
-    }
-    int64_t grid = (int64_t)h->sm_count * per_sm;
-    if (grid > need) grid = need;
-    h->round_grid = (int)grid;
+    h->round_grid = (int)(need < kRoundGridCap ? need : kRoundGridCap);
   }
+  const size_t n_groups = (size_t)((h->round_grid + kFinishGroup - 1) / kFinishGroup);
   HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_partials,
                            sizeof(double) * 2 * kMaxDevices * (size_t)h->round_grid));
-  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_ticket, sizeof(unsigned int)));
-  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int), h->stream));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_group_partials, sizeof(double) * 2 * kMaxDevices * n_groups));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_ticket, sizeof(unsigned int) * (1 + n_groups)));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int) * (1 + n_groups), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
   return launch_init(h);
@@ -427,6 +398,7 @@ int hadfl_destroy(hadfl_handle *h) {
   cudaFree(h->d_ticket);
   cudaFree(h->d_stats);
   cudaFree(h->d_round_partials);
+  cudaFree(h->d_round_group_partials);
   cudaFree(h->d_round_ticket);
   if (h->backup_stream) cudaStreamSynchronize(h->backup_stream);
   cudaFree(h->d_backup);
@@ -751,16 +723,27 @@ int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t
     g_noalloc_sms[dev] = sms;
     g_noalloc_ptr[dev] = (unsigned char *)p;
   }
+  // Both buffers must be device memory of the current device: anything else (a host pointer, another
+  // GPU's memory) would turn into a memory fault inside the kernel instead of an error status.
+  // cudaPointerGetAttributes allocates nothing.
+  {
+    const void *ptrs[2] = {w, out_stats};
+    for (const void *q : ptrs) {
+      cudaPointerAttributes at;
+      if (cudaPointerGetAttributes(&at, q) != cudaSuccess) {
+        cudaGetLastError();
+        return HADFL_ERR_INVALID;
+      }
+      if ((at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) || at.device != dev)
+        return HADFL_ERR_INVALID;
+    }
+  }
   unsigned int *ticket = (unsigned int *)g_noalloc_ptr[dev];
   double *partials = (double *)(g_noalloc_ptr[dev] + 256);
   // Same grid rule as the handle's statistics launch, capped by what the scratch holds.
-  const int64_t pack_e = dtype == HADFL_DTYPE_BF16 ? 8 : 4;
-  const int64_t packs = (n_params + pack_e - 1) / pack_e;
-  const int64_t chunks = (packs + kThreads * kStatsU - 1) / (kThreads * kStatsU);
-  int64_t lanes = ((int64_t)g_noalloc_sms[dev] * 8 + n_devices - 1) / n_devices;
-  if (lanes > chunks) lanes = chunks;
-  if (lanes * n_devices > HADFL_NOALLOC_MAX_BLOCKS) lanes = HADFL_NOALLOC_MAX_BLOCKS / n_devices;
+  const int64_t lanes = stats_lanes_for(g_noalloc_sms[dev], n_devices, n_params, dtype, HADFL_NOALLOC_MAX_BLOCKS);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
+  cudaGetLastError();  // an error left behind by earlier, unrelated work is not this call's
   // The array keeps the previous call's contents: the ticket must start at zero.
   if (cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream) != cudaSuccess) return HADFL_ERR_CUDA;
   const unsigned blocks = (unsigned)(lanes * n_devices);
@@ -773,6 +756,13 @@ int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t
         (const float *)w, row_stride_elems, n_params, n_devices, ref_device, (int)lanes, partials,
         ticket, out_stats);
   return cudaGetLastError() == cudaSuccess ? HADFL_OK : HADFL_ERR_CUDA;
+}
+
+int64_t hadfl_stats_grid_lanes(int32_t sm_count, int32_t n_devices, int64_t n_params, int32_t dtype,
+                               int64_t max_blocks) {
+  if (sm_count < 1 || n_devices < 1 || n_devices > HADFL_MAX_DEVICES || n_params < 1 || max_blocks < 0) return 0;
+  if (dtype != HADFL_DTYPE_FP32 && dtype != HADFL_DTYPE_BF16) return 0;
+  return stats_lanes_for(sm_count, n_devices, n_params, dtype, max_blocks);
 }
 
 int hadfl_read_params(hadfl_handle *h, int32_t id, float *dst, int64_t count) {
@@ -875,6 +865,7 @@ int hadfl_synchronize(hadfl_handle *h) {
 int hadfl_last_cuda_error(const hadfl_handle *h) { return h ? h->last_cuda_error : 0; }
 uint64_t hadfl_launch_count(const hadfl_handle *h) { return h ? h->launches : 0; }
 int64_t hadfl_row_stride(const hadfl_handle *h) { return h ? h->stride : 0; }
+int32_t hadfl_round_grid(const hadfl_handle *h) { return h ? h->round_grid : 0; }
 
 int hadfl_selection_probs(const double *x, const uint8_t *avail, int32_t n, double *out_P) {
   if (!x || !out_P || n < 1 || n > HADFL_MAX_DEVICES) return HADFL_ERR_INVALID;

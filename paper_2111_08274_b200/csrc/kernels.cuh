@@ -219,9 +219,11 @@ __device__ __forceinline__ float sfu_cos(float x) {
 }
 
 // -2 ln(1 - t) by its series, for t = 1 - u0 = (~x0 + 0.5) 2^-32 < 2^-10, times `scale2`:
-// 2t + t^2 + (2/3) t^3 (the next term, t^4/2, is below 2^-31 relative).  Kept out of line so that
-// the common path pays one compare and an untaken branch for it.
-__device__ __noinline__ float r2_next_to_one(uint32_t x0, float scale2) {
+// 2t + t^2 + (2/3) t^3 (the next term, t^4/2, is below 2^-31 relative).  Only reached from a rarely
+// taken branch (one combined test per step), so the common path pays a compare and an untaken
+// branch for it; inlined there, because a real call inside the step loop makes the compiler shuffle
+// the live registers around every call site (about one instruction per step on average).
+__device__ __forceinline__ float r2_next_to_one(uint32_t x0, float scale2) {
   const float t = fmaf(__uint2float_rn(~x0), 0x1p-32f, 0x1p-33f);
   return scale2 * (t * fmaf(t, fmaf(t, 0.66666667f, 1.0f), 2.0f));
 }
@@ -704,6 +706,59 @@ __device__ __forceinline__ void finish_by_last_block(const double *__restrict__ 
   if (threadIdx.x == 0) *ticket = 0u;
 }
 
+// Two-level variant for grids of many blocks (the fused round).  Blocks are grouped in runs of
+// kFinishGroup consecutive block indices.  The block that draws a group's last ticket sums that
+// group's partials[t][first block of the group ...] in block order -> group_partials[t][group]
+// and draws the launch's ticket; the block that draws the last of those sums the group sums in
+// group order and hands them to `emit`.  Each of the two sums has a fixed order that does not
+// depend on which block happens to compute it, so the result is reproducible; no block waits for
+// another; all tickets are back at zero when the launch ends.
+constexpr int kFinishGroup = 128;
+
+template <typename Emit>
+__device__ __forceinline__ void finish_two_level(const double *__restrict__ partials,
+                                                 double *__restrict__ group_partials, int n_vals,
+                                                 unsigned int *__restrict__ group_tickets,
+                                                 unsigned int *__restrict__ ticket, bool *s_last,
+                                                 Emit emit) {
+  const int n_blocks = (int)gridDim.x;
+  const int n_groups = (n_blocks + kFinishGroup - 1) / kFinishGroup;
+  const int g = (int)blockIdx.x / kFinishGroup;
+  const int g_first = g * kFinishGroup;
+  const int g_size = min(kFinishGroup, n_blocks - g_first);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) *s_last = (atomicAdd(group_tickets + g, 1u) == (unsigned)g_size - 1u);
+  __syncthreads();
+  if (!*s_last) return;
+  __threadfence();
+  for (int t = warp; t < n_vals; t += kThreads / 32) {
+    const double *src = partials + (int64_t)t * n_blocks + g_first;
+    double s = 0.0;
+    for (int l = lane; l < g_size; l += 32) s += __ldcg(src + l);
+    s = warp_sum(s);
+    if (lane == 0) group_partials[(int64_t)t * n_groups + g] = s;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    group_tickets[g] = 0u;
+    *s_last = (atomicAdd(ticket, 1u) == (unsigned)n_groups - 1u);
+  }
+  __syncthreads();
+  if (!*s_last) return;
+  __threadfence();
+  for (int t = warp; t < n_vals; t += kThreads / 32) {
+    const double *src = group_partials + (int64_t)t * n_groups;
+    double s = 0.0;
+    for (int l = lane; l < n_groups; l += 32) s += __ldcg(src + l);
+    s = warp_sum(s);
+    if (lane == 0) emit(t, s);
+  }
+  if (threadIdx.x == 0) *ticket = 0u;
+}
+
 // ------------------------------------------------------------------------------------------
 // K3: per-replica squared norm and squared distance to a reference replica.
 // Block b works on row b % N and on the chunks (b / N), (b / N) + lanes, ...; a chunk is
@@ -801,10 +856,20 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 // Parameters and momentum come out bit-identical to K1 followed by K2 (and the broadcast); the
 // aggregate is never re-read from memory, so a round moves 16 bytes per (device, parameter)
 // instead of 20 + 8k/N.
-// Grid: persistent, grid-stride over packs.  Row sums: one shuffle per row and pack, then a
-// shared-memory slot owned by the thread (fp32); at the end a butterfly over each half-warp, a
-// fixed-order fp64 sum over warps -> partials[value][block]; last-ticket block finishes.
-// Deterministic.  Dynamic shared memory: n * kThreads floats.
+//
+// Grid: one block per chunk of kThreads packs, up to a cap beyond which the blocks stride over
+// the chunks; the hardware block scheduler then balances the SMs (a one-wave persistent grid ends
+// with a partly filled last pass and keeps all blocks in the same phase of their rows: measured
+// 7-15 % slower with several steps per device).  The chunk loop's trip count depends on the block
+// index only, so control flow and every row descriptor read inside it are uniform across the
+// block - with a per-thread loop bound the compiler re-read the descriptors through indexed
+// constant loads in every step (+7 instructions per step).  Lanes beyond the end of the vector
+// (live = 0) take part in everything: their loads return zeros, their stores store nothing, and
+// what they compute is zeroed before it is summed.
+// Row sums: one shuffle per row and pack, then a shared-memory slot owned by the thread (fp32); at
+// the end of the block, per row, a fixed-order sum over the warps and a butterfly over each
+// half-warp (fp64) -> partials[value][block]; two-level last-ticket finish.  Deterministic.
+// Dynamic shared memory: n * kThreads floats.  64 registers: four resident blocks per SM.
 // ------------------------------------------------------------------------------------------
 struct RoundArgs {
   int32_t n;          // rows visited = all N devices: [0, k) selected in draw order, then the rest
@@ -828,49 +893,42 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
   *slot += keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
 }
 
-// MINB: resident blocks per SM the kernel is compiled for (3: 75 registers, 4: 64 registers with a
-// few bytes of spills).  With bf16 parameters a row is 48 bytes per thread or less and the fourth
-// block buys more bytes in flight than the tighter register budget costs (+10 % at one step per
-// device); with fp32 parameters three blocks are faster per element, and four are used only where
-// the larger wave saves a whole pass of the persistent loop (the host decides per handle).
-template <typename WT, typename MT, typename Gen, int E, int RM, int MINB>
-__global__ void __launch_bounds__(kThreads, MINB)
+constexpr int kRoundBlocksPerSM = 4;
+
+template <typename WT, typename MT, typename Gen, int E, int RM>
+__global__ void __launch_bounds__(kThreads, kRoundBlocksPerSM)
 k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
-        StepConsts k, double *__restrict__ partials, unsigned int *__restrict__ ticket,
+        StepConsts k, double *__restrict__ partials, double *__restrict__ group_partials,
+        unsigned int *__restrict__ group_tickets, unsigned int *__restrict__ ticket,
         float *__restrict__ out) {
   constexpr int kWarps = kThreads / 32;
-  extern __shared__ float s_acc[];                   // [a.n][kThreads]: per-thread row sums
-  __shared__ double s_sum[kWarps][2 * kMaxDevices];  // [warp][2 * visit index + which]
+  extern __shared__ float s_acc[];  // [a.n][kThreads]: per-thread row sums
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int j = 0; j < a.n; ++j) s_acc[j * kThreads + threadIdx.x] = 0.f;
 
   const int64_t n_packs = (n_params + E - 1) / E;
-  // Whole warps iterate together (the row sums use a shuffle): the pack count is rounded up to a
-  // multiple of 32; lanes beyond the end carry live = 0, load and store nothing, and add zeros.
-  const int64_t n_packs_padded = (n_packs + 31) / 32 * 32;
-
-  for (int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x; p < n_packs_padded;
-       p += (int64_t)gridDim.x * kThreads) {
-    // Lanes beyond the end (live = 0) take part in everything: their loads return zeros, their
-    // stores store nothing, and what they compute is zeroed before it is summed - so control flow
-    // stays uniform across the warp (the step loop's trip count is a launch parameter).
+  const int64_t n_chunks = (n_packs + kThreads - 1) / kThreads;
+  for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+    const int64_t p = chunk * kThreads + threadIdx.x;
     const int live = live_of(n_params, p, E);
     const GroupProducts<E / 4> gp(p);
     char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
     char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
-    float acc[E];
-#pragma unroll
-    for (int i = 0; i < E; ++i) acc[i] = 0.f;
 
-    auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
+    // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
+    // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
+    // 0).  fp32 values are updated in the registers they were loaded into.
+    auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
+      RawPack<WT, E> rw;
       ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-      if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
-    };
-    // One row: its steps, then its part in the aggregation / synchronisation and in the sums.
-    auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
       const bool stepped = a.r[j].steps > 0;
       if (stepped) {
+        RawPack<MT, E> rm;
+        ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
+        float mv[E];
+        unpack(rw, wv);
+        unpack(rm, mv);
         sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
         if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
         st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
@@ -880,92 +938,81 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
 #pragma unroll
           for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
         }
-      }
-      if (j < a.k) {  // a selected device, visited in draw order: fold into the aggregate
-        const float aj = a.a[j];
-        if (j == 0) {
-#pragma unroll
-          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(aj, wv[i]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
-        }
-        if (j == a.k - 1) {
-          float n2 = 0.f;
-#pragma unroll
-          for (int i = 0; i < E; ++i) {
-            acc[i] = as_stored(acc[i], w);
-            n2 = fmaf(acc[i], acc[i], n2);
-          }
-          // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
-          if (a.k > 1 || a.r[0].steps > 0)
-            for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
-          add_row_sums(s_acc, j, n2, 0.f, lane);  // one value for all selected devices
-        }
-      } else {  // another device: keep its own model, or receive the aggregate
-        if (a.write_all == 1) {
-#pragma unroll
-          for (int i = 0; i < E; ++i) wv[i] = acc[i];
-        } else if (a.write_all == 2) {
-#pragma unroll
-          for (int i = 0; i < E; ++i)
-            wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
-        }
-        if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-        float n2 = 0.f, d2 = 0.f;
-#pragma unroll
-        for (int i = 0; i < E; ++i) {
-          const float d = wv[i] - acc[i];
-          n2 = fmaf(wv[i], wv[i], n2);
-          d2 = fmaf(d, d, d2);
-        }
-        add_row_sums(s_acc, j, n2, d2, lane);
-      }
-    };
-    // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
-    auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
-      if constexpr (sizeof(WT) == 4) {
-        body(j, rw.v, rm.v);
-      } else if constexpr (sizeof(MT) == 4) {
-        float wv[E];
-        unpack(rw, wv);
-        body(j, wv, rm.v);
       } else {
-        float wv[E], mv[E];
         unpack(rw, wv);
-        unpack(rm, mv);  // only used when the row runs steps (the momentum is loaded only then)
-        body(j, wv, mv);
       }
+      return stepped;
     };
-    // No prefetch of the next row (as in K1): the registers it would take cost a resident block,
-    // and one more block per SM hides the row loads better than a prefetch.
-    RawPack<WT, E> rw;
-    RawPack<MT, E> rm;
-    zero_raw(rw);
-    zero_raw(rm);
-    for (int j = 0; j < a.n; ++j) {
-      load(j, rw, rm);
-      visit(j, rw, rm);
+
+    // ---- the selected devices in draw order: acc = a_0 w_0, then acc = fma(a_j, w_j, acc)
+    float acc[E];
+    {
+      float wv[E];
+      row_after_steps(0, wv);
+      const float a0 = a.a[0];
+#pragma unroll
+      for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
+    }
+    for (int j = 1; j < a.k; ++j) {
+      float wv[E];
+      row_after_steps(j, wv);
+      const float aj = a.a[j];
+#pragma unroll
+      for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
+    }
+    {
+      float n2 = 0.f;
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        acc[i] = as_stored(acc[i], w);
+        n2 = fmaf(acc[i], acc[i], n2);
+      }
+      // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
+      if (a.k > 1 || a.r[0].steps > 0)
+        for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
+      add_row_sums(s_acc, a.k - 1, n2, 0.f, lane);  // one value for all selected devices
+    }
+    // ---- the other devices: keep their own model, or receive the aggregate
+    for (int j = a.k; j < a.n; ++j) {
+      float wv[E];
+      const bool stepped = row_after_steps(j, wv);
+      if (a.write_all == 1) {
+#pragma unroll
+        for (int i = 0; i < E; ++i) wv[i] = acc[i];
+      } else if (a.write_all == 2) {
+#pragma unroll
+        for (int i = 0; i < E; ++i)
+          wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
+      }
+      if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+      float n2 = 0.f, d2 = 0.f;
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        const float d = wv[i] - acc[i];
+        n2 = fmaf(wv[i], wv[i], n2);
+        d2 = fmaf(d, d, d2);
+      }
+      add_row_sums(s_acc, j, n2, d2, lane);
     }
   }
-  // ---- block: fold the per-thread slots (lower half-warps hold norms, upper halves distances)
-  for (int j = a.k - 1; j < a.n; ++j) {
-    float v = s_acc[j * kThreads + threadIdx.x];
-#pragma unroll
-    for (int off = 8; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-    if ((lane & 15) == 0) s_sum[warp][2 * j + (lane >> 4)] = (double)v;
-  }
+  // ---- block: sum the per-thread slots of every visit index j >= k - 1.  Warp w takes the visit
+  // indices k - 1 + w, k - 1 + w + 8, ...: each lane adds the slots of the threads that share its
+  // lane index (one per warp, in warp order; lower half-warps hold norms, upper halves distances),
+  // then a butterfly over the half-warp finishes the two sums.
   __syncthreads();
-  // partials[value][block]; value = 2 * visit index + which
-  const int n_vals = 2 * a.n;
-  if ((int)threadIdx.x < n_vals && (int)threadIdx.x >= 2 * (a.k - 1)) {
-    double s = 0.0;
-    for (int wi = 0; wi < kWarps; ++wi) s += s_sum[wi][threadIdx.x];
-    partials[(int64_t)threadIdx.x * gridDim.x + blockIdx.x] = s;
+  for (int j = a.k - 1 + warp; j < a.n; j += kWarps) {
+    float v = 0.f;
+#pragma unroll
+    for (int wi = 0; wi < kWarps; ++wi) v += s_acc[j * kThreads + wi * 32 + lane];
+    double d = (double)v;
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) d += __shfl_xor_sync(0xFFFFFFFFu, d, off);
+    // partials[value][block]; value = 2 * visit index + which
+    if ((lane & 15) == 0) partials[(int64_t)(2 * j + (lane >> 4)) * gridDim.x + blockIdx.x] = d;
   }
   const int n_dev = a.n, ksel = a.k;
-  finish_by_last_block(partials + (int64_t)2 * (ksel - 1) * gridDim.x, n_vals - 2 * (ksel - 1),
-                       (int)gridDim.x, ticket, &s_last, [&](int t, double sum) {
+  finish_two_level(partials + (int64_t)2 * (ksel - 1) * gridDim.x, group_partials, 2 * (n_dev - ksel + 1),
+                   group_tickets, ticket, &s_last, [&](int t, double sum) {
     const int j = ksel - 1 + (t >> 1), which = t & 1;
     if (j == ksel - 1) {  // the selected devices share one norm and are at distance 0
       for (int q = 0; q < ksel; ++q) out[which * n_dev + a.r[q].row] = which ? 0.f : (float)sum;

@@ -96,11 +96,17 @@ def shrink(w: Workload, n_params: int, rounds: Optional[int] = None) -> Workload
 
 
 def by_name(name: str) -> Workload:
+    """c1, c2, c3, c4_k{2,8,16}, c5_p{16..27}_{fp32,bf16}[_het]."""
     table = {"c1": c1, "c2": c2, "c3": c3}
     if name in table:
         return table[name]()
     if name.startswith("c4"):
         return c4(int(name.split("k")[-1])) if "k" in name else c4()
+    if name.startswith("c5_p"):
+        parts = name.split("_")
+        if len(parts) >= 3 and parts[2] in ("fp32", "bf16"):
+            return c5(int(parts[1][1:]), dtype=1 if parts[2] == "bf16" else 0,
+                      hetero=len(parts) > 3 and parts[3] == "het")
     raise KeyError(name)
 
 
@@ -110,13 +116,27 @@ def random_rows(n_rows: int, n_params: int, seed: int, std: float = 0.05) -> np.
     return (rng.standard_normal((n_rows, n_params)) * std).astype(np.float32)
 
 
-def sample_groups(n_params: int, n_random: int, edge: int, seed: int) -> np.ndarray:
-    """Sorted, distinct 4-column group indices: the first and last `edge` groups of the vector
-    plus `n_random` groups drawn uniformly from the rest."""
+def sample_groups(n_params: int, n_random: int, edge: int, seed: int, around=(), halo: int = 64) -> np.ndarray:
+    """Sorted, distinct 4-column group indices: the first and last `edge` groups of the vector,
+    `n_random` groups drawn uniformly from the rest, and the `halo` groups on either side of every
+    group index listed in `around` (e.g. where one pass of a grid ends and the next begins)."""
     n_groups = (n_params + 3) // 4
     if n_groups <= 2 * edge + n_random:
         return np.arange(n_groups, dtype=np.uint32)
     rng = np.random.default_rng(seed)
     mid = rng.choice(np.arange(edge, n_groups - edge), size=n_random, replace=False)
-    out = np.concatenate([np.arange(edge), mid, np.arange(n_groups - edge, n_groups)])
-    return np.unique(out).astype(np.uint32)
+    parts = [np.arange(edge), mid, np.arange(n_groups - edge, n_groups)]
+    for g in around:
+        parts.append(np.arange(max(0, int(g) - halo), min(n_groups, int(g) + halo)))
+    return np.unique(np.concatenate(parts)).astype(np.uint32)
+
+
+def pass_boundaries(n_params: int, threads_per_pass, cols_per_thread: int = 8):
+    """Group indices at which a grid of `threads_per_pass` threads, each holding `cols_per_thread`
+    columns, starts a new pass over a vector of n_params columns - for every entry of
+    threads_per_pass.  Only used to aim column samples at those seams."""
+    out = []
+    for t in threads_per_pass:
+        step = int(t) * cols_per_thread // 4
+        out.extend(range(step, (n_params + 3) // 4, step))
+    return out

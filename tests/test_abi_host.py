@@ -93,3 +93,23 @@ def test_no_handle_is_rejected_not_crashed(lib):
     assert lib.hadfl_synchronize(None) == binding.ERR_INVALID
     assert lib.hadfl_destroy(None) == binding.OK
     assert lib.hadfl_init(None, None) == binding.ERR_INVALID
+
+
+def test_statistics_grid_rule_and_its_cap(lib):
+    """The grid rule of the statistics kernel as a host function: one wave of 8 blocks per SM split
+    over the rows, at most one block per 16 KB chunk of a row, and the block cap that bounds the
+    scratch of hadfl_stats_noalloc (which a 148-SM GPU never reaches, a larger one would)."""
+    from paper_2111_08274_b200 import binding
+    f = binding.hadfl_stats_grid_lanes
+    big = 1 << 30
+    assert f(148, 8, big) == 148                       # 1184 resident blocks over 8 rows
+    assert f(148, 32, big) == 37
+    assert f(148, 32, big, 0, 2048) == 37              # the cap does not bind on 148 SMs
+    assert f(148, 1, big, 0, 2048) == 1184
+    assert f(148, 8, 4096) == 1 and f(148, 8, 4097) == 2 and f(148, 8, 1) == 1   # one block per 4096 fp32 values
+    assert f(148, 8, 8192, 1) == 1 and f(148, 8, 8193, 1) == 2                   # ... or 8192 bf16 values
+    for sms, n in ((300, 8), (300, 32), (1024, 3), (257, 1)):                    # beyond 256 SMs the cap binds
+        lanes = f(sms, n, big, 0, 2048)
+        assert lanes * n <= 2048 < (lanes + 1) * n, (sms, n, lanes)
+        assert f(sms, n, big) * n >= 8 * sms
+    assert f(0, 8, big) == 0 and f(148, 33, big) == 0 and f(148, 8, 0) == 0 and f(148, 8, big, 2) == 0

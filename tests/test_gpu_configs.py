@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_common import TOL_REL, assert_close_params, bf16_ulp, require_gpu
+from gpu_common import compare_sample, require_gpu, run_and_compare
 from oracle_driver import make_sim, oracle_round
 from paper_2111_08274_b200 import runtime, workloads
 
@@ -22,60 +22,11 @@ def _gpu():
     require_gpu()
 
 
-def columns_of(groups, n_params):
-    cols = (4 * groups.astype(np.int64)[:, None] + np.arange(4)[None, :]).reshape(-1)
-    return cols, cols < n_params
-
-
-def compare_sample(arena, sim, groups, what):
-    wl = arena.wl
-    cols, live = columns_of(groups, wl.n_params)
-    idx = torch.from_numpy(np.where(live, cols, 0)).to(arena.device)
-    worst = 0.0
-    for i in range(wl.n_devices):
-        got = arena.w[i, idx].float().cpu().numpy()[live]
-        want = sim.read_cols(i)[live]
-        if wl.dtype == 0:
-            worst = max(worst, assert_close_params(got, want, "%s w[%d]" % (what, i)))
-        else:
-            # A rounding decision that went the other way leaves a difference of one bf16 step of the
-            # value at that time, which persists while the value itself moves on: bound it by two
-            # steps at the largest magnitude in the row, and require such elements to be rare.
-            assert np.abs(got - want).max() <= 2 * bf16_ulp(np.abs(want).max()), (what, i)
-            assert np.mean(got != want) < 0.01, (what, i)
-        gm = arena.m[i, idx].cpu().numpy()[live]
-        # momentum sees the generator's error directly (not scaled by lr); with bf16 storage a
-        # moved rounding of w also enters through weight decay
-        m_tol = wl.grad_std * 1e-5 / (1.0 - wl.momentum) + (wl.weight_decay * 0.004 / (1.0 - wl.momentum) if wl.dtype else 0.0)
-        assert np.abs(gm - sim.read_momentum_cols(i)[live]).max() <= m_tol, (what, i)
-    return worst
-
-
-def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=(), fused=False):
-    arena = runtime.Arena(wl)
-    sim = make_sim(oracle, wl, groups)
-    full = groups is None
-    g = np.arange((wl.n_params + 3) // 4, dtype=np.uint32) if full else groups
-    worst = 0.0
-    for r in range(wl.rounds):
-        sel = arena.run_round_fused(r) if fused else arena.run_round(r)
-        want_sel = oracle_round(sim, wl, r)
-        assert np.array_equal(sel, want_sel), "round %d: selection %s != %s" % (r, sel, want_sel)
-        v, s = arena.h.get_versions()
-        ov, os_ = sim.get_versions()
-        assert np.array_equal(v, ov) and np.array_equal(s, os_), "round %d: counters differ" % r
-        if r in check_rounds or r == wl.rounds - 1:
-            worst = max(worst, compare_sample(arena, sim, g, "%s round %d" % (wl.name, r)))
-        if full and (r in stats_rounds or r == wl.rounds - 1):
-            n2, d2 = arena.h.stats_read()
-            wn2, wd2 = sim.stats(int(sel[0]))
-            assert np.allclose(n2, wn2, rtol=1e-5) and np.allclose(d2, wd2, rtol=1e-5, atol=1e-12)
-    n2, d2 = arena.h.stats_read()
-    assert np.all(np.isfinite(n2)) and np.all(d2 >= 0) and d2[int(sel[0])] == 0.0
-    launches = arena.h.launch_count()
-    arena.close()
-    print("%s: %d rounds ok, max err / max|x| = %.2e, %d launches" % (wl.name, wl.rounds, worst, launches))
-    return worst
+def seams(wl):
+    """Column groups where a one-wave grid of 3 or 4 blocks of 256 threads per SM (148 SMs, 8
+    columns per thread) would start its next pass: a fault confined to the seam between passes, or
+    to a partly filled last pass, would sit there."""
+    return workloads.pass_boundaries(wl.n_params, [148 * 3 * 256, 148 * 4 * 256])
 
 
 def test_c1_full_arena_every_round(oracle):
@@ -99,13 +50,13 @@ def test_c2_full_size_fused_round_sampled_columns(oracle):
     """The launch configuration the benchmark times: the whole round of the full-size workload in
     one hadfl_round call per round."""
     wl = workloads.c2()
-    groups = workloads.sample_groups(wl.n_params, 30_000, 1024, seed=22)
+    groups = workloads.sample_groups(wl.n_params, 65_536, 1024, seed=22, around=seams(wl))   # 2^18 random columns
     run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24), fused=True)
 
 
 def test_c3_full_size_fused_round_sampled_columns(oracle):
     wl = workloads.c3()
-    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=33)
+    groups = workloads.sample_groups(wl.n_params, 12_000, 1024, seed=33, around=seams(wl))
     run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 10, 49), fused=True)
 
 
@@ -131,20 +82,22 @@ def test_c3_full_size_sampled_columns(oracle):
     run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 10, 49))
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("k", [2, 8, 16])
-def test_c4_full_size_sampled_columns(oracle, k):
+def test_c4_full_size_sampled_columns(oracle, k, fused):
     wl = workloads.c4(k)
-    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=4 + k)
-    run_and_compare(oracle, wl, groups, check_rounds=(0, 9))
+    groups = workloads.sample_groups(wl.n_params, 6_000, 1024, seed=4 + k, around=seams(wl), halo=16)
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9), fused=fused)
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("log2_p", range(16, 28))
-def test_c5_bandwidth_sweep_sizes(oracle, log2_p, dtype):
+def test_c5_bandwidth_sweep_sizes(oracle, log2_p, dtype, fused):
     for hetero in (False, True):
         wl = workloads.c5(log2_p, dtype=dtype, hetero=hetero)
-        groups = workloads.sample_groups(wl.n_params, 256, 128, seed=log2_p)
-        run_and_compare(oracle, wl, groups, check_rounds=(0, 4, 99))
+        groups = workloads.sample_groups(wl.n_params, 256, 128, seed=log2_p, around=seams(wl), halo=4)
+        run_and_compare(oracle, wl, groups, check_rounds=(0, 4, 99), fused=fused)
 
 
 @pytest.mark.parametrize("dtype", [0, 1])

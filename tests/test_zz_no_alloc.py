@@ -2,7 +2,8 @@
 memory (their memory belongs to another allocator, or an allocation's device-wide synchronisation
 is unaffordable where they run).  It takes no handle, keeps its scratch in a fixed array inside the
 library and works on raw device pointers.  Checked here against hadfl_stats on the same arena, on
-two calls in a row (the second one finds the first one's leftovers in the shared scratch).
+two calls in a row (the second one finds the first one's leftovers in the shared scratch), and
+against the CPU oracle's double-precision sums.
 
 This file is collected last on purpose: if it fails under `pytest -x`, every other test has run."""
 import numpy as np
@@ -10,6 +11,7 @@ import pytest
 import torch
 
 from gpu_common import require_gpu
+from oracle_driver import make_sim
 from paper_2111_08274_b200 import binding, runtime, workloads
 from paper_2111_08274_b200.workloads import Workload
 
@@ -33,10 +35,11 @@ def noalloc_stats(arena, ref, out):
 
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("n,P", [(4, 100_003), (16, 1_500_001), (32, 4099), (1, 7)])
-def test_matches_hadfl_stats_on_two_calls_in_a_row(n, P, dtype):
+def test_matches_hadfl_stats_on_two_calls_in_a_row(oracle, n, P, dtype):
     wl = Workload("na", n, P, min(2, n), 1, "fixed", tuple(1 + i % 3 for i in range(n)),
                   grad_std=1e-2, dtype=dtype, seed=workloads.BASE_SEED + 77)
     arena = runtime.Arena(wl)
+    sim = make_sim(oracle, wl)          # its replicas are overwritten with the arena's values below
     out = torch.full((2 * n,), -1.0, dtype=torch.float32, device=arena.device)   # caller's buffer
     arena.h.local_step(wl.device_ids(), wl.steps_for_round(0), wl.lr)
     for call, ref in enumerate((0, n - 1)):
@@ -45,6 +48,12 @@ def test_matches_hadfl_stats_on_two_calls_in_a_row(n, P, dtype):
         assert np.allclose(got_n2, want_n2, rtol=1e-5, atol=0), (call, got_n2, want_n2)
         assert np.allclose(got_d2, want_d2, rtol=1e-5, atol=0), (call, got_d2, want_d2)
         assert got_d2[ref] == 0.0
+        # the oracle sums, in double, the very values the arena holds (read back bit for bit)
+        for i in range(n):
+            sim.write_params(i, arena.h.read_params(i))
+        on2, od2 = sim.stats(ref)
+        assert np.allclose(got_n2, on2, rtol=1e-5, atol=0), (call, got_n2, on2)
+        assert np.allclose(got_d2, od2, rtol=1e-5, atol=1e-30), (call, got_d2, od2)
         # the arena moves on between the two calls, so stale scratch could not go unnoticed
         arena.h.local_step(wl.device_ids(), wl.steps_for_round(1), wl.lr)
     arena.close()
@@ -64,6 +73,18 @@ def test_limits_and_bad_arguments_are_refused_without_touching_the_output():
     assert f(None, 0, 4, 4099, st, 0, out.data_ptr(), s) == binding.ERR_INVALID
     assert f(w + 4, 0, 4, 4099, st, 0, out.data_ptr(), s) == binding.ERR_INVALID
     assert f(w, 0, 4, 4099, st, 0, None, s) == binding.ERR_INVALID
+    # buffers that are not device memory of the current GPU are refused on the host, not in the kernel
+    host_w = np.zeros(4 * st, dtype=np.float32)
+    host_out = np.zeros(8, dtype=np.float32)
+    aligned = host_w.ctypes.data + (-host_w.ctypes.data) % 16
+    assert f(aligned, 0, 1, 7, 8, 0, out.data_ptr(), s) == binding.ERR_INVALID
+    assert f(w, 0, 4, 4099, st, 0, host_out.ctypes.data, s) == binding.ERR_INVALID
+    pinned = torch.zeros(8, dtype=torch.float32).pin_memory()
+    assert f(w, 0, 4, 4099, st, 0, pinned.data_ptr(), s) == binding.ERR_INVALID
+    assert f(w, 0, 4, 4099, st, 0, out.data_ptr(), s) == binding.OK      # and a later good call still works
+    torch.cuda.synchronize()
+    assert torch.all(out != -1.0)
+    out.fill_(-1.0)
     torch.cuda.synchronize()
     assert torch.all(out == -1.0)
     arena.close()
