@@ -69,7 +69,7 @@ ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to 
 #   peak = SMs x 4 sub-partitions x SM clock / max(PIPE_CYCLES)      [element-steps per second]
 # with the SM clock sampled during the timed region.  "issue" is the warp scheduler's issue slot
 # (one instruction per cycle); the integer multiplies of Philox occupy the FMA-heavy pipe.
-PIPE_CYCLES_PER_ELEM_STEP = {"issue": 0.6046, "fmaheavy": 0.6046, "fmalite": 0.0, "alu": 0.0, "xu": 0.0}
+PIPE_CYCLES_PER_ELEM_STEP = {"fmaheavy": 0.6141, "issue": 0.6046, "xu": 0.5000, "alu": 0.3572, "fmalite": 0.2667}
 PIPE_CYCLES_SOURCE = "profiles/k_local_step_pipes_N8_P4M.md"
 
 # DRAM bytes per unit of work moved by one launch, from the ncu captures summarised under profiles/
@@ -78,8 +78,8 @@ PIPE_CYCLES_SOURCE = "profiles/k_local_step_pipes_N8_P4M.md"
 # small capture up to 126 MB of written lines are still dirty in L2 when the kernel ends and are
 # not counted.  Unit: (device, parameter) for the round, the local update and the statistics, one
 # element of a selected row for the aggregation.  None = not captured for the kernel as it stands.
-NCU_DRAM_READ_PER_UNIT = {"round": None, "local_step": 8.00, "aggregate": 4.00, "stats": 4.00}
-NCU_DRAM_WRITE_PER_UNIT = {"round": None, "local_step": 6.29, "aggregate": 0.58, "stats": 0.11}
+NCU_DRAM_READ_PER_UNIT = {"round": 8.00, "local_step": 8.00, "aggregate": 4.00, "stats": 4.00}
+NCU_DRAM_WRITE_PER_UNIT = {"round": 6.13, "local_step": 6.12, "aggregate": 0.30, "stats": 0.004}
 NCU_DRAM_SOURCE = "profiles/kernels_small_case_N8_P4M.md"
 
 
