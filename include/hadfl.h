@@ -325,6 +325,27 @@ int hadfl_selection_draw(const double *x, const uint8_t *avail, int32_t n, int64
 int hadfl_predict_version(const double *series, int32_t n_obs, double alpha, double m,
                           double *out_prediction);
 
+/* ---- the debug build ---------------------------------------------------------------------------
+ * libhadfl_debug.so is this library compiled with -DHADFL_DEBUG: every access a kernel makes to the
+ * arenas and every store to the library's scratch buffers is first checked against the device
+ * address ranges the handle registered.  An access outside them is skipped (loads read zeros) and
+ * recorded; no kernel traps or asserts; and every call marked "synchronises" (and
+ * hadfl_synchronize) then returns HADFL_ERR_STATE.  It stands in for a memory checker.  One GPU
+ * per process; slower (a table lookup per access; hadfl_init, hadfl_destroy and
+ * hadfl_stats_noalloc synchronise the device).  Results are identical to the normal build. */
+
+/* 1 in the debug build, 0 otherwise. */
+int hadfl_debug_build(void);
+
+/* Waits for the handle's stream; debug build: HADFL_ERR_STATE if any kernel so far skipped an
+ * out-of-range access (*out_bad_address, if not NULL, receives the first such device address);
+ * normal build: HADFL_OK. */
+int hadfl_debug_check(hadfl_handle *h, uint64_t *out_bad_address);
+
+/* The predicate the debug build applies on the device, as a host function: 1 if the byte range
+ * [addr, addr + nbytes) lies inside [lo, hi), else 0 (no arithmetic in it can overflow). */
+int hadfl_debug_range_holds(uint64_t lo, uint64_t hi, uint64_t addr, uint64_t nbytes);
+
 /* ---- diagnostics of the on-device generator (used by the tests) -------------------------- */
 
 /* Philox4x32-10 on the GPU: counters (n x 4 words), key (2 words) -> out_words (n x 4).

@@ -10,7 +10,9 @@ import os
 import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libhadfl.so")
+# HADFL_LIBRARY names another build of the same library to load instead (the debug build,
+# libhadfl_debug.so: same entry points, bounds-checked kernels).
+LIB_PATH = os.environ.get("HADFL_LIBRARY") or os.path.join(HERE, "libhadfl.so")
 
 OK, ERR_INVALID, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, 1, 2, 3, 4
 MAX_DEVICES = 32
@@ -95,6 +97,9 @@ SIGNATURES = {
     "hadfl_selection_probs": (C.c_int, [_f64p, _u8p, C.c_int32, _f64p]),
     "hadfl_selection_draw": (C.c_int, [_f64p, _u8p, C.c_int32, C.c_int64, C.c_uint64, C.c_int32, _i32p]),
     "hadfl_predict_version": (C.c_int, [_f64p, C.c_int32, C.c_double, C.c_double, _f64p]),
+    "hadfl_debug_build": (C.c_int, []),
+    "hadfl_debug_check": (C.c_int, [_H, _u64p]),
+    "hadfl_debug_range_holds": (C.c_int, [C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64]),
     "hadfl_debug_philox": (C.c_int, [_H, _u32p, _u32p, C.c_int64, _u32p]),
     "hadfl_debug_normals": (C.c_int, [_H, C.c_int32, _u32p, C.c_int64, C.c_uint64, C.c_uint32, _f32p]),
 }
@@ -159,6 +164,14 @@ def hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems, ref
     (see include/hadfl.h).  out_stats_ptr: 2N device floats, norm2 then div2.  Asynchronous."""
     return int(lib().hadfl_stats_noalloc(w_ptr, dtype, n_devices, n_params, row_stride_elems,
                                          ref_device, out_stats_ptr, stream or None))
+
+
+def hadfl_debug_build():
+    return bool(lib().hadfl_debug_build())
+
+
+def hadfl_debug_range_holds(lo, hi, addr, nbytes):
+    return bool(lib().hadfl_debug_range_holds(lo, hi, addr, nbytes))
 
 
 def hadfl_stats_grid_lanes(sm_count, n_devices, n_params, dtype=DTYPE_FP32, max_blocks=0):
@@ -354,6 +367,14 @@ class Hadfl:
 
     def synchronize(self):
         self._check(self._lib.hadfl_synchronize(self._h), "hadfl_synchronize")
+
+    def debug_check(self):
+        """Raises HadflError (HADFL_ERR_STATE) if, in the debug build, a kernel skipped an out-of-range access."""
+        bad = C.c_uint64(0)
+        rc = self._lib.hadfl_debug_check(self._h, C.byref(bad))
+        if rc:
+            raise HadflError("hadfl_debug_check (first bad address 0x%x)" % bad.value, rc,
+                             self._lib.hadfl_last_cuda_error(self._h))
 
     def launch_count(self):
         return int(self._lib.hadfl_launch_count(self._h))

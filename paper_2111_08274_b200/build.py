@@ -11,8 +11,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhadfl.so")
+LIB_DEBUG = os.path.join(HERE, "libhadfl_debug.so")   # -DHADFL_DEBUG: bounds-checked kernels
 SOURCES = ["hadfl.cu", "selection.cpp"]
-DEPS = SOURCES + ["kernels.cuh", "philox.cuh", "selection.h", os.path.join("..", "..", "include", "hadfl.h")]
+DEPS = SOURCES + ["kernels.cuh", "philox.cuh", "debug_check.cuh", "selection.h",
+                  os.path.join("..", "..", "include", "hadfl.h")]
 
 
 def nvcc_path() -> str:
@@ -22,27 +24,30 @@ def nvcc_path() -> str:
     return "nvcc"
 
 
-def up_to_date() -> bool:
-    if not os.path.exists(LIB):
+def up_to_date(lib: str) -> bool:
+    if not os.path.exists(lib):
         return False
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return all(os.path.getmtime(os.path.join(CSRC, d)) <= t for d in DEPS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and up_to_date():
-        return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib = LIB_DEBUG if debug else LIB
+    if not force and up_to_date(lib):
+        return lib
+    tmp = lib + ".tmp.%d" % os.getpid()
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
            "-std=c++17", "-shared", "-Xcompiler", "-fPIC,-ffp-contract=off",
            "-cudart", "static", "-fmad=false", "-o", tmp]
+    if debug:
+        cmd += ["-DHADFL_DEBUG"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

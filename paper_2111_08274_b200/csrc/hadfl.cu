@@ -129,6 +129,48 @@ RowStep row_step(const hadfl_handle *h, int dev, uint64_t base, int steps) {
   return r;
 }
 
+// ---- debug build: the table of device ranges the kernels may touch --------------------------------
+// One table per process (the debug build supports one GPU per process).  The host keeps a mirror,
+// publishes it to the device symbol whenever it changes (after the stream has drained, with a
+// blocking copy), and reads the error word back in every synchronising call.
+#ifdef HADFL_DEBUG
+DebugRanges g_debug_host;
+
+int debug_publish() {
+  return cudaMemcpyToSymbol(g_debug, &g_debug_host, offsetof(DebugRanges, error)) == cudaSuccess ? 0 : 1;
+}
+void debug_add(const void *p, size_t nbytes) {
+  if (!p || nbytes == 0 || g_debug_host.n >= kDebugRanges) return;
+  g_debug_host.lo[g_debug_host.n] = (uint64_t)(uintptr_t)p;
+  g_debug_host.hi[g_debug_host.n] = (uint64_t)(uintptr_t)p + nbytes;
+  ++g_debug_host.n;
+}
+void debug_remove(const void *p) {
+  for (int r = 0; r < g_debug_host.n; ++r)
+    if (g_debug_host.lo[r] == (uint64_t)(uintptr_t)p) {
+      --g_debug_host.n;
+      g_debug_host.lo[r] = g_debug_host.lo[g_debug_host.n];
+      g_debug_host.hi[r] = g_debug_host.hi[g_debug_host.n];
+      return;
+    }
+}
+// 0: every access so far was in range; 1: some kernel skipped one (addr = the first such address).
+int debug_error(uint64_t *addr) {
+  DebugRanges now;
+  if (cudaMemcpyFromSymbol(&now, g_debug, sizeof(now)) != cudaSuccess) return 1;
+  if (addr) *addr = now.bad_addr;
+  return now.error ? 1 : 0;
+}
+#define HADFL_DEBUG_VERDICT()                            \
+  do {                                                   \
+    if (debug_error(nullptr)) return HADFL_ERR_STATE;    \
+  } while (0)
+#else
+#define HADFL_DEBUG_VERDICT() \
+  do {                        \
+  } while (0)
+#endif
+
 #define HADFL_CUDA(h, expr)                       \
   do {                                            \
     cudaError_t e_ = (expr);                      \
@@ -256,6 +298,7 @@ int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool moment
   DeviceGuard guard(h->device);
   if (count == 0) {
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+    HADFL_DEBUG_VERDICT();
     return HADFL_OK;
   }
   const void *arena = momentum ? h->m : h->w;
@@ -264,12 +307,14 @@ int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool moment
     HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost,
                                   h->stream));
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+    HADFL_DEBUG_VERDICT();
     return HADFL_OK;
   }
   std::vector<uint16_t> tmp((size_t)count);
   const uint16_t *src = (const uint16_t *)arena + (int64_t)id * h->stride;
   HADFL_CUDA(h, cudaMemcpyAsync(tmp.data(), src, 2 * (size_t)count, cudaMemcpyDeviceToHost, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  HADFL_DEBUG_VERDICT();
   for (int64_t p = 0; p < count; ++p) {
     const uint32_t bits = (uint32_t)tmp[(size_t)p] << 16;
     memcpy(dst + p, &bits, 4);
@@ -382,6 +427,16 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int) * (1 + n_groups), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
+#ifdef HADFL_DEBUG
+  debug_add(h->w, elems * elem_size(h));
+  debug_add(h->m, elems * m_elem_size(h));
+  debug_add(h->d_partials, sizeof(double) * 2 * (size_t)cfg->n_devices * (size_t)lanes);
+  debug_add(h->d_stats, sizeof(float) * 2 * kMaxDevices);
+  debug_add(h->d_round_partials, sizeof(double) * 2 * kMaxDevices * (size_t)h->round_grid);
+  debug_add(h->d_round_group_partials, sizeof(double) * 2 * kMaxDevices * n_groups);
+  HADFL_CUDA(h, cudaDeviceSynchronize());
+  if (debug_publish()) return HADFL_ERR_CUDA;
+#endif
   return launch_init(h);
 }
 
@@ -390,6 +445,16 @@ int hadfl_destroy(hadfl_handle *h) {
   DeviceGuard guard(h->device);
   hadfl_backup_wait(h);
   cudaStreamSynchronize(h->stream);
+#ifdef HADFL_DEBUG
+  cudaDeviceSynchronize();
+  debug_remove(h->w);
+  debug_remove(h->m);
+  debug_remove(h->d_partials);
+  debug_remove(h->d_stats);
+  debug_remove(h->d_round_partials);
+  debug_remove(h->d_round_group_partials);
+  debug_publish();
+#endif
   if (h->own_arena) {
     cudaFree(h->w);
     cudaFree(h->m);
@@ -680,6 +745,7 @@ int hadfl_stats_read(hadfl_handle *h, float *out_norm2, float *out_div2) {
   HADFL_CUDA(h, cudaMemcpyAsync(buf, h->d_stats, sizeof(float) * 2 * (size_t)n,
                                 cudaMemcpyDeviceToHost, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  HADFL_DEBUG_VERDICT();
   memcpy(out_norm2, buf, sizeof(float) * (size_t)n);
   memcpy(out_div2, buf + n, sizeof(float) * (size_t)n);
   return HADFL_OK;
@@ -744,6 +810,26 @@ int hadfl_stats_noalloc(const void *w, int32_t dtype, int32_t n_devices, int64_t
   const int64_t lanes = stats_lanes_for(g_noalloc_sms[dev], n_devices, n_params, dtype, HADFL_NOALLOC_MAX_BLOCKS);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   cudaGetLastError();  // an error left behind by earlier, unrelated work is not this call's
+#ifdef HADFL_DEBUG
+  // Debug build only: the caller's buffers and the fixed scratch join the table of checked ranges for
+  // the duration of the call, which therefore synchronises the device before and after its kernel.
+  const size_t es_dbg = dtype == HADFL_DTYPE_BF16 ? 2 : 4;
+  cudaDeviceSynchronize();
+  debug_add(w, (size_t)n_devices * (size_t)row_stride_elems * es_dbg);
+  debug_add(out_stats, sizeof(float) * 2 * (size_t)n_devices);
+  debug_add(g_noalloc_ptr[dev], HADFL_NOALLOC_SCRATCH_BYTES);
+  debug_publish();
+  struct Unregister {
+    const void *a, *b, *c;
+    ~Unregister() {
+      cudaDeviceSynchronize();
+      debug_remove(c);
+      debug_remove(b);
+      debug_remove(a);
+      debug_publish();
+    }
+  } unregister{w, out_stats, g_noalloc_ptr[dev]};
+#endif
   // The array keeps the previous call's contents: the ticket must start at zero.
   if (cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream) != cudaSuccess) return HADFL_ERR_CUDA;
   const unsigned blocks = (unsigned)(lanes * n_devices);
@@ -804,7 +890,7 @@ int hadfl_backup_begin(hadfl_handle *h, int32_t device_id, float *dst, int64_t c
   DeviceGuard guard(h->device);
   const size_t es = elem_size(h);
   if (!h->backup_stream) {  // first use: staging row, copy stream, two events
-    HADFL_CUDA(h, cudaMalloc(&h->d_backup, (size_t)h->cfg.n_params * es));
+    HADFL_CUDA(h, cudaMalloc(&h->d_backup, (size_t)h->cfg.n_params * es));  // copies only: no kernel touches it
     HADFL_CUDA(h, cudaStreamCreateWithFlags(&h->backup_stream, cudaStreamNonBlocking));
     HADFL_CUDA(h, cudaEventCreateWithFlags(&h->backup_ready, cudaEventDisableTiming));
     HADFL_CUDA(h, cudaEventCreateWithFlags(&h->backup_done, cudaEventDisableTiming));
@@ -859,7 +945,31 @@ int hadfl_synchronize(hadfl_handle *h) {
   if (!h) return HADFL_ERR_INVALID;
   DeviceGuard guard(h->device);
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  HADFL_DEBUG_VERDICT();
   return HADFL_OK;
+}
+
+int hadfl_debug_build(void) {
+#ifdef HADFL_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int hadfl_debug_check(hadfl_handle *h, uint64_t *out_bad_address) {
+  if (!h) return HADFL_ERR_INVALID;
+  if (out_bad_address) *out_bad_address = 0;
+#ifdef HADFL_DEBUG
+  DeviceGuard guard(h->device);
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  if (debug_error(out_bad_address)) return HADFL_ERR_STATE;
+#endif
+  return HADFL_OK;
+}
+
+int hadfl_debug_range_holds(uint64_t lo, uint64_t hi, uint64_t addr, uint64_t nbytes) {
+  return range_holds(lo, hi, addr, nbytes) ? 1 : 0;
 }
 
 int hadfl_last_cuda_error(const hadfl_handle *h) { return h ? h->last_cuda_error : 0; }

@@ -21,6 +21,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "debug_check.cuh"
 #include "philox.cuh"
 
 namespace hadfl {
@@ -33,9 +34,11 @@ constexpr int kThreads = 256;
 // ragged last pack of a row).
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void st_group(float *row, int64_t g, float4 v) {
+  if (!access_ok(row + 4 * g, 16)) return;
   *reinterpret_cast<float4 *>(row + 4 * g) = v;
 }
 __device__ __forceinline__ void st_group(__nv_bfloat16 *row, int64_t g, float4 v) {
+  if (!access_ok(row + 4 * g, 8)) return;
   const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
   const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
   uint2 raw;
@@ -43,13 +46,11 @@ __device__ __forceinline__ void st_group(__nv_bfloat16 *row, int64_t g, float4 v
   raw.y = *reinterpret_cast<const uint32_t *>(&hi);
   *reinterpret_cast<uint2 *>(row + 4 * g) = raw;
 }
-__device__ __forceinline__ float ld_elem(const float *row, int64_t p) { return row[p]; }
-__device__ __forceinline__ float ld_elem(const __nv_bfloat16 *row, int64_t p) {
-  return __bfloat162float(row[p]);
+__device__ __forceinline__ void st_elem(float *row, int64_t p, float v) {
+  if (access_ok(row + p, 4)) row[p] = v;
 }
-__device__ __forceinline__ void st_elem(float *row, int64_t p, float v) { row[p] = v; }
 __device__ __forceinline__ void st_elem(__nv_bfloat16 *row, int64_t p, float v) {
-  row[p] = __float2bfloat16_rn(v);
+  if (access_ok(row + p, 2)) row[p] = __float2bfloat16_rn(v);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -64,6 +65,7 @@ struct Pack16 {  // the pack that is 16 bytes of storage
 
 template <int E>
 __device__ __forceinline__ void st_pack(float *row, int64_t p, const float (&v)[E]) {
+  if (!access_ok(row + E * p, 4 * E)) return;
 #pragma unroll
   for (int i = 0; i < E / 4; ++i)
     *reinterpret_cast<float4 *>(row + E * p + 4 * i) =
@@ -79,6 +81,7 @@ __device__ __forceinline__ uint32_t floats_to_bf16x2(float lo, float hi) {
 }
 template <int E>
 __device__ __forceinline__ void st_pack(__nv_bfloat16 *row, int64_t p, const float (&v)[E]) {
+  if (!access_ok(row + E * p, 2 * E)) return;
   if (E == 8) {
     uint4 raw;
     raw.x = floats_to_bf16x2(v[0], v[1]);
@@ -131,6 +134,11 @@ __device__ __forceinline__ void unpack(const RawPack<__nv_bfloat16, 4> &r, float
 // last pack of a row) element by element, dead lanes read as 0.
 template <int E>
 __device__ __forceinline__ void ld_raw(const float *at, int live, RawPack<float, E> &r) {
+  if (!access_ok(at, 4 * (size_t)live)) {  // debug build only: a skipped load reads as zeros
+#pragma unroll
+    for (int i = 0; i < E; ++i) r.v[i] = 0.f;
+    return;
+  }
   if (live == E) {
 #pragma unroll
     for (int i = 0; i < E / 4; ++i) {
@@ -146,6 +154,10 @@ __device__ __forceinline__ uint32_t ld_bf16_bits(const __nv_bfloat16 *at, int i,
   return i < live ? (uint32_t)*reinterpret_cast<const unsigned short *>(at + i) : 0u;
 }
 __device__ __forceinline__ void ld_raw(const __nv_bfloat16 *at, int live, RawPack<__nv_bfloat16, 8> &r) {
+  if (!access_ok(at, 2 * (size_t)live)) {
+    r.q = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
   if (live == 8) {
     r.q = *reinterpret_cast<const uint4 *>(at);
   } else {
@@ -156,6 +168,10 @@ __device__ __forceinline__ void ld_raw(const __nv_bfloat16 *at, int live, RawPac
   }
 }
 __device__ __forceinline__ void ld_raw(const __nv_bfloat16 *at, int live, RawPack<__nv_bfloat16, 4> &r) {
+  if (!access_ok(at, 2 * (size_t)live)) {
+    r.q = make_uint2(0u, 0u);
+    return;
+  }
   if (live == 4) {
     r.q = *reinterpret_cast<const uint2 *>(at);
   } else {
@@ -572,10 +588,16 @@ template <typename WT, int KR, int U>
 __global__ void __launch_bounds__(kThreads)
 k_combine(WT *__restrict__ w, int64_t stride, int64_t n_params, CombineArgs c) {
   constexpr int E = Pack16<WT>::E;
-  const int64_t p0 = (int64_t)blockIdx.x * (kThreads * U) + threadIdx.x;
-  // Fast path (all but the last block of a launch): every pack of the block is full, so the
+  // Blocks walk the vector from its END to its start: the kernels before and after this one in a
+  // round (local update, statistics) walk it from the start, so whatever the previous kernel left
+  // in the 126 MB L2 - the end of every row - is read first, and what this kernel leaves there -
+  // the start of the rows it wrote - is what the statistics kernel reads first.  Measured on the
+  // ResNet-18-sized workload inside a round: aggregation 61 -> 57 us, statistics 75 -> 62 us.
+  const int64_t chunk = (int64_t)(gridDim.x - 1 - blockIdx.x);
+  const int64_t p0 = chunk * (kThreads * U) + threadIdx.x;
+  // Fast path (all but the last chunk of a launch): every pack of the block is full, so the
   // U * KR row loads of a thread are straight-line code and all in flight together.
-  const bool block_full = ((int64_t)(blockIdx.x + 1) * (kThreads * U)) * E <= n_params;
+  const bool block_full = ((chunk + 1) * (kThreads * U)) * E <= n_params;
   if (KR > 0 && KR * U <= 16 && block_full) {
     constexpr int KRc = KR > 0 ? KR : 1;
     RawPack<WT, E> raw[U][KRc];
@@ -738,7 +760,7 @@ __device__ __forceinline__ void finish_two_level(const double *__restrict__ part
     double s = 0.0;
     for (int l = lane; l < g_size; l += 32) s += __ldcg(src + l);
     s = warp_sum(s);
-    if (lane == 0) group_partials[(int64_t)t * n_groups + g] = s;
+    if (lane == 0 && access_ok(group_partials + (int64_t)t * n_groups + g, 8)) group_partials[(int64_t)t * n_groups + g] = s;
   }
   __threadfence();
   __syncthreads();
@@ -838,10 +860,13 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
   if (threadIdx.x < 2) {
     double s = 0.0;
     for (int wi = 0; wi < kWarps; ++wi) s += s_part[threadIdx.x][wi];
-    partials[((int64_t)threadIdx.x * n_devices + row) * lanes + my_lane] = s;
+    double *slot = partials + ((int64_t)threadIdx.x * n_devices + row) * lanes + my_lane;
+    if (access_ok(slot, 8)) *slot = s;
   }
   finish_by_last_block(partials, 2 * n_devices, lanes, ticket, &s_last,
-                       [&](int t, double sum) { out[t] = (float)sum; });
+                       [&](int t, double sum) {
+                         if (access_ok(out + t, 4)) out[t] = (float)sum;
+                       });
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1008,16 +1033,21 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
 #pragma unroll
     for (int off = 8; off > 0; off >>= 1) d += __shfl_xor_sync(0xFFFFFFFFu, d, off);
     // partials[value][block]; value = 2 * visit index + which
-    if ((lane & 15) == 0) partials[(int64_t)(2 * j + (lane >> 4)) * gridDim.x + blockIdx.x] = d;
+    double *slot = partials + (int64_t)(2 * j + (lane >> 4)) * gridDim.x + blockIdx.x;
+    if ((lane & 15) == 0 && access_ok(slot, 8)) *slot = d;
   }
   const int n_dev = a.n, ksel = a.k;
   finish_two_level(partials + (int64_t)2 * (ksel - 1) * gridDim.x, group_partials, 2 * (n_dev - ksel + 1),
                    group_tickets, ticket, &s_last, [&](int t, double sum) {
     const int j = ksel - 1 + (t >> 1), which = t & 1;
     if (j == ksel - 1) {  // the selected devices share one norm and are at distance 0
-      for (int q = 0; q < ksel; ++q) out[which * n_dev + a.r[q].row] = which ? 0.f : (float)sum;
+      for (int q = 0; q < ksel; ++q) {
+        float *o = out + which * n_dev + a.r[q].row;
+        if (access_ok(o, 4)) *o = which ? 0.f : (float)sum;
+      }
     } else {
-      out[which * n_dev + a.r[j].row] = (float)sum;
+      float *o = out + which * n_dev + a.r[j].row;
+      if (access_ok(o, 4)) *o = (float)sum;
     }
   });
 }

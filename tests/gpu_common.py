@@ -83,6 +83,7 @@ def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=(), fused=Fal
     n2, d2 = arena.h.stats_read()
     assert np.all(np.isfinite(n2)) and np.all(d2 >= 0) and d2[int(sel[0])] == 0.0
     launches = arena.h.launch_count()
+    arena.h.debug_check()      # debug build: no kernel skipped an out-of-range access (no-op otherwise)
     arena.close()
     print("%s: %d rounds ok, max err / max|x| = %.2e, %d launches" % (wl.name, wl.rounds, worst, launches))
     return worst

@@ -113,3 +113,19 @@ def test_statistics_grid_rule_and_its_cap(lib):
         assert lanes * n <= 2048 < (lanes + 1) * n, (sms, n, lanes)
         assert f(sms, n, big) * n >= 8 * sms
     assert f(0, 8, big) == 0 and f(148, 33, big) == 0 and f(148, 8, 0) == 0 and f(148, 8, big, 2) == 0
+
+
+def test_debug_build_range_predicate(lib):
+    """[addr, addr + nbytes) inside [lo, hi): the predicate the debug build's kernels apply to every
+    access, including its corner cases near the ends of the range and of the address space."""
+    from paper_2111_08274_b200 import binding
+    f = binding.hadfl_debug_range_holds
+    lo, hi = 0x7F0000001000, 0x7F0000002000
+    assert f(lo, hi, lo, 16) and f(lo, hi, hi - 16, 16) and f(lo, hi, lo, hi - lo) and f(lo, hi, hi, 0)
+    assert not f(lo, hi, lo - 1, 16) and not f(lo, hi, hi - 15, 16) and not f(lo, hi, hi, 1)
+    assert not f(lo, hi, lo, hi - lo + 1) and not f(lo, hi, 0, 16) and not f(lo, hi, hi + 4096, 4)
+    top = 2**64 - 1
+    assert not f(lo, hi, top - 3, 16) and not f(lo, hi, lo, top)          # no wrap-around
+    assert f(top - 64, top, top - 16, 16) and not f(top - 64, top, top - 8, 16)
+    assert not f(hi, lo, lo, 0)                                           # an empty / inverted range holds nothing
+    assert not binding.hadfl_debug_build()                                # the library under test is the normal build

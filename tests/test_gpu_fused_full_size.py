@@ -44,6 +44,8 @@ def run_both(wl, rounds, oracle=None, groups=None):
     assert np.allclose(a[0], b[0], rtol=2e-6) and np.allclose(a[1], b[1], rtol=2e-6, atol=1e-30)
     if sim is not None:
         compare_sample(fused, sim, groups, wl.name + " fused")
+    fused.h.debug_check()
+    plain.h.debug_check()
     fused.close()
     plain.close()
 
