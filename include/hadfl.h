@@ -135,6 +135,13 @@ int hadfl_select(hadfl_handle *h, int64_t round, const double *versions, uint64_
 /* Eq. 8 itself: out_P[i] = P(i) (0 for unavailable devices).  Host only. */
 int hadfl_select_probs(hadfl_handle *h, const double *versions, double *out_P);
 
+/* Eq. 8 on the versions the devices WILL have once device_ids[j] has run steps[j] more local steps
+ * (each listed device's version grows by its step count; the others keep theirs): the probabilities
+ * from which hadfl_round(device_ids, steps, ..., versions = NULL) draws its selection, for callers
+ * that want to log them beside a fused round.  n distinct ids, steps >= 0.  Host only. */
+int hadfl_select_probs_after(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
+                             double *out_P);
+
 /* Partial aggregation, Eq. 5 / Algorithm 1 "partial synchronization", fused with the write-back:
  *     acc = a_0 * w[selected[0]];  acc = fma(a_j, w[selected[j]], acc), j = 1..k-1;
  *     w[selected[j]] = acc for all j          (one kernel, every element touched once)

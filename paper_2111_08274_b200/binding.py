@@ -66,6 +66,7 @@ SIGNATURES = {
     "hadfl_local_step": (C.c_int, [_H, _i32p, _i32p, C.c_int32, C.c_float]),
     "hadfl_select": (C.c_int, [_H, C.c_int64, _f64p, C.c_uint64, C.c_int32, _i32p]),
     "hadfl_select_probs": (C.c_int, [_H, _f64p, _f64p]),
+    "hadfl_select_probs_after": (C.c_int, [_H, _i32p, _i32p, C.c_int32, _f64p]),
     "hadfl_aggregate": (C.c_int, [_H, _i32p, C.c_int32, _f64p]),
     "hadfl_aggregation_weights": (C.c_int, [_H, _i32p, C.c_int32, _f64p, _f32p]),
     "hadfl_broadcast": (C.c_int, [_H, C.c_int32, _i32p, C.c_int32]),
@@ -246,6 +247,16 @@ class Hadfl:
         out = np.empty(self.n_devices, dtype=np.float64)
         self._check(self._lib.hadfl_select_probs(self._h, _p(v, C.c_double), _p(out, C.c_double)),
                     "hadfl_select_probs")
+        return out
+
+    def select_probs_after(self, device_ids, steps):
+        ids, st = _arr(device_ids, np.int32), _arr(steps, np.int32)
+        if len(ids) != len(st):
+            raise HadflError("hadfl_select_probs_after", ERR_INVALID)
+        out = np.empty(self.n_devices, dtype=np.float64)
+        self._check(self._lib.hadfl_select_probs_after(self._h, _p(ids, C.c_int32), _p(st, C.c_int32),
+                                                       len(ids), _p(out, C.c_double)),
+                    "hadfl_select_probs_after")
         return out
 
     def aggregate(self, selected, versions=None):

@@ -536,6 +536,19 @@ int hadfl_select_probs(hadfl_handle *h, const double *versions, double *out_P) {
   return selection_probs(x, h->avail, h->cfg.n_devices, out_P) ? HADFL_OK : HADFL_ERR_INVALID;
 }
 
+int hadfl_select_probs_after(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
+                             double *out_P) {
+  if (!h || !out_P || !steps || !distinct_ids(h, device_ids, n)) return HADFL_ERR_INVALID;
+  double x[kMaxDevices];
+  for (int i = 0; i < h->cfg.n_devices; ++i) x[i] = (double)h->version[i];
+  for (int j = 0; j < n; ++j) {
+    if (steps[j] < 0) return HADFL_ERR_INVALID;
+    x[device_ids[j]] = (double)(h->version[device_ids[j]] + (uint32_t)steps[j]);
+  }
+  for (int i = 0; i < h->cfg.n_devices; ++i) x[i] *= h->cfg.version_scale;
+  return selection_probs(x, h->avail, h->cfg.n_devices, out_P) ? HADFL_OK : HADFL_ERR_INVALID;
+}
+
 int hadfl_aggregation_weights(hadfl_handle *h, const int32_t *selected, int32_t k,
                               const double *versions, float *out_a) {
   if (!h || !out_a || !distinct_ids(h, selected, k)) return HADFL_ERR_INVALID;

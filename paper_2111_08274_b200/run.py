@@ -65,9 +65,7 @@ def main(argv=None):
                     h.integrate(int(sel[0]), others, wl.sync_beta)
             h.stats_enqueue(int(sel[0]))
         else:
-            v_now, _ = h.get_versions()
-            probs = h.select_probs(planned if planned is not None
-                                   else (v_now + steps.astype(np.uint32)).astype(np.float64))
+            probs = h.select_probs(planned) if planned is not None else h.select_probs_after(arena.ids, steps)
             sel = h.round(arena.ids, steps, wl.lr, r, wl.k, arena.select_seed, versions=planned,
                           sync_all=sync)
         end.record(arena.stream)

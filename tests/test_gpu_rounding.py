@@ -75,6 +75,41 @@ def test_local_step_without_noise_is_bit_exact(oracle, P, m_dtype, rounding):
     assert np.array_equal(h.get_versions()[1], sim.get_versions()[1])
 
 
+@pytest.mark.parametrize("m_dtype,rounding", [(0, 0)] + MODES)
+def test_a_call_that_crosses_a_multiple_of_two_to_the_32_steps_rounds_where_it_is_split(oracle, m_dtype, rounding):
+    """The kernels take the high word of a device's step index as fixed per launch, so a call whose
+    step counter crosses a multiple of 2^32 runs as two launches - and with bf16 storage the values
+    are rounded at the end of each.  The documented behaviour is therefore that of the SAME steps
+    given as two calls (up to the crossing, beyond it): pinned here bit for bit, without gradient
+    noise, against the oracle driven that way; the oracle's single call (one rounding) may differ
+    from it by at most one bf16 step."""
+    n, P = 3, 4099
+    wl = wl_of(n, P, m_dtype, rounding, grad_std=0.0, weight_decay=0.3, momentum=0.9)
+    h, two_calls, one_call = binding.Hadfl.from_workload(wl), make_sim(oracle, wl), make_sim(oracle, wl)
+    rows = workloads.random_rows(n, P, seed=91)
+    mom = workloads.random_rows(n, P, seed=92, std=0.01)
+    for sim in (two_calls, one_call):
+        load_rows(h, sim, rows, mom)
+    start = np.array([2**32 - 2, 7, 2**33 - 1], dtype=np.uint64)
+    for x in (h, two_calls, one_call):
+        x.set_versions(step_counts=start)
+    ids, steps = [0, 1, 2], [5, 3, 4]
+    h.local_step(ids, steps, 0.05)
+    two_calls.local_step(ids, [2, 3, 1], 0.05)          # up to the crossing (device 1 does not cross)
+    two_calls.local_step([0, 2], [3, 3], 0.05)          # beyond it
+    one_call.local_step(ids, steps, 0.05)
+    assert np.array_equal(h.get_versions()[1], two_calls.get_versions()[1])
+    assert np.array_equal(h.get_versions()[1], one_call.get_versions()[1])
+    for i in range(n):
+        got_w, got_m = h.read_params(i), h.read_momentum(i)
+        assert np.array_equal(got_w, two_calls.read_params(i)), i
+        assert np.array_equal(got_m, two_calls.read_momentum(i)), i
+        once = one_call.read_params(i)
+        assert np.abs(got_w - once).max() <= bf16_ulp(np.abs(once).max()), i
+    assert np.array_equal(h.read_params(1), one_call.read_params(1))       # no crossing, no split
+    h.destroy()
+
+
 def test_stochastic_rounding_moves_where_nearest_even_stalls(oracle):
     """Weight decay only, lr wd = 1e-3 < half a bf16 spacing: nearest-even storage never moves,
     stochastic storage follows the oracle bit for bit (whose mean is pinned to the closed form)."""
