@@ -1,7 +1,8 @@
 """Benchmark of the HADFL round hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
-                    [--min-seconds 0.5] [--no-sweep] [--no-cpu-baseline]
+                    [--min-seconds 0.5] [--sweep default|full|none] [--no-cpu-baseline]
+    python bench.py --table saved_line.json                               (markdown tables of its sweep)
     python bench.py --profile-case [--pc-fused] [--pc-steps 1,8] ...      (target of ncu captures)
 
 A "step" is one round of the whole hot path over one synthetic workload: local update of every
@@ -309,14 +310,21 @@ def measure_case(wl, rounds, peak, frac_key, warmup=3):
     evf = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(rounds)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
-    start.record()
     for i in range(rounds):
         a, b = evf[i]
         a.record(); arena.run_round_fused(r + i); b.record()
-    end.record()
     torch.cuda.synchronize()
     fused_ms = float(np.median([a.elapsed_time(b) for a, b in evf]))
-    fused_wall_ms = start.elapsed_time(end) / rounds
+    r += rounds
+    # rounds/s with 8 rounds enqueued per library call (hadfl_rounds): small vectors then show the
+    # kernel and not the per-call overhead of the caller, while the launch queue stays shallow
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(0, 2 * rounds, 8):
+        arena.run_rounds_fused(r + i, min(8, 2 * rounds - i))
+    end.record()
+    torch.cuda.synchronize()
+    fused_wall_ms = start.elapsed_time(end) / (2 * rounds)
     grid = h.round_grid()
     arena.close()
     nbytes = {"local_step": N * P * 2 * (ew + em), "aggregate": 2 * k * P * ew, "stats": N * P * ew,
@@ -335,19 +343,98 @@ def measure_case(wl, rounds, peak, frac_key, warmup=3):
     return res
 
 
-def run_sweep(peak, frac_key, rounds=12):
-    """The metric against P (bandwidth sweep) and the two larger CNN-sized workloads."""
+def measure_sync(wl, peak, frac_key, reps=30):
+    """Global synchronisation from device 0 to the N - k others: overwrite and beta-mix."""
     import torch
+    from paper_2111_08274_b200 import runtime
+    arena = runtime.Arena(wl)
+    h = arena.h
+    ew = 2 if wl.dtype else 4
+    dst = np.arange(wl.k, wl.n_devices, dtype=np.int32)
+    out = {"workload": wl.name, "N": wl.n_devices, "P": wl.n_params, "receivers": len(dst),
+           "storage": "bf16" if wl.dtype else "fp32", "kernels": {}}
+    for name, call, nbytes in (("broadcast", lambda: h.broadcast(0, dst), (1 + len(dst)) * wl.n_params * ew),
+                               ("integrate", lambda: h.integrate(0, dst, 0.5), (1 + 2 * len(dst)) * wl.n_params * ew)):
+        for _ in range(3):
+            call()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            call()
+        b.record()
+        torch.cuda.synchronize()
+        out["kernels"][name] = gbs_entry(nbytes, a.elapsed_time(b) / reps, peak, frac_key)
+    arena.close()
+    return out
+
+
+def sweep_cases(which):
+    """default: the bandwidth sweep at five sizes, both storages, one step per device and step ratios
+    1,1,2,2,4,4,8,8, plus the VGG-16- and ResNet-50-sized workloads.  full: every size 2^16 .. 2^27, all
+    five workloads with k in {2, 8, 16}, the ResNet-18 size at one step per device, and the
+    reduced-precision variants (bf16 momentum, stochastic rounding)."""
+    from dataclasses import replace
     cases = [workloads.c3(), workloads.c4(8)]
+    sizes = (20, 22, 24, 26, 27)
+    if which == "full":
+        cases = [workloads.c1(), workloads.c2(), workloads.c3(), workloads.c4(2), workloads.c4(8), workloads.c4(16),
+                 workloads.Workload("c2_steps1", 8, 11_173_962, 4, 50, "fixed", (1,) * 8, seed=workloads.BASE_SEED + 2)]
+        sizes = tuple(range(16, 28))
     for dtype in (0, 1):
         for hetero in (False, True):
-            for lp in (20, 22, 24, 26, 27):
+            for lp in sizes:
                 cases.append(workloads.c5(lp, dtype=dtype, hetero=hetero))
+    if which == "full":
+        for hetero in (False, True):
+            for m_dtype, rounding in ((0, 1), (1, 0), (1, 1)):
+                base = workloads.c5(25, dtype=1, hetero=hetero)
+                name = base.name + ("_m16" if m_dtype else "") + ("_sr" if rounding else "")
+                cases.append(replace(base, name=name, m_dtype=m_dtype, rounding=rounding))
+    return cases
+
+
+def run_sweep(peak, frac_key, which="default", rounds=12):
+    """The metric against P (bandwidth sweep) and the larger CNN-sized workloads."""
+    import torch
     out = []
-    for wl in cases:
+    for wl in sweep_cases(which):
         out.append(measure_case(wl, rounds, peak, frac_key))
         torch.cuda.empty_cache()
-    return out
+    sync = []
+    if which == "full":
+        for wl in (workloads.c2(), workloads.c3(), workloads.c4(8), workloads.c5(25, dtype=1)):
+            sync.append(measure_sync(wl, peak, frac_key))
+            torch.cuda.empty_cache()
+    return out, sync
+
+
+def print_tables(path):
+    """Markdown tables of the sweep carried by a saved JSON line of this benchmark."""
+    with open(path) as f:
+        line = json.loads(f.read().strip().splitlines()[-1])
+    sw = line["sweep"]
+    peak = sw["peak_gbs"]
+    key = "frac_of_%s_hbm" % sw["peak_kind"]
+
+    def cell(k):
+        return "%.1f | %.0f (%.0f / %.0f)" % (k["avg_ms"] * 1e3, k["achieved_gbs"], 100 * k[key], 100 * k["frac_of_8TBs"])
+    print("GB/s = algorithmic bytes / time; percentages: of the %s %.0f GB/s / of the nominal 8000 GB/s.\n" % (sw["peak_kind"], peak))
+    print("| workload | N | P | k | storage | mean steps | K1 µs | K1 GB/s (% meas / % 8T) | K2 µs | K2 GB/s (%/%) | K3 µs | K3 GB/s (%/%) "
+          "| separate calls rounds/s | fused `hadfl_round` µs | fused GB/s (%/%) | fused rounds/s | G element-steps/s |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for p in sw["points"]:
+        ks = p["kernels"]
+        print("| %s | %d | %d | %d | %s | %.2f | %s | %s | %s | %.0f | %s | %.0f | %.0f |" % (
+            p["workload"], p["N"], p["P"], p["k"], p["storage"], p["mean_steps_per_device"], cell(ks["local_step"]),
+            cell(ks["aggregate"]), cell(ks["stats"]), p["separate_calls_rounds_per_s"], cell(ks["round"]),
+            p["rounds_per_s"], ks["round"]["gelem_steps_per_s"]))
+    if sw.get("sync"):
+        print("\n| workload | N | P | receivers | storage | broadcast µs | GB/s (%/%) | integrate µs | GB/s (%/%) |")
+        print("|---|---|---|---|---|---|---|---|---|")
+        for p in sw["sync"]:
+            print("| %s | %d | %d | %d | %s | %s | %s |" % (p["workload"], p["N"], p["P"], p["receivers"], p["storage"],
+                                                         cell(p["kernels"]["broadcast"]), cell(p["kernels"]["integrate"])))
 
 
 # ---- our arm ---------------------------------------------------------------------------------------
@@ -587,10 +674,13 @@ def run_ours(args, wl):
     arena.close()
     del host_model
     torch.cuda.empty_cache()
-    if rank == 0 and world == 1 and not args.no_sweep:
+    if rank == 0 and world == 1 and args.sweep != "none":
+        points, sync = run_sweep(peak, frac_key, args.sweep)
         line["sweep"] = {"what": "fused round (rounds/s, one hadfl_round call per round, CUDA events) and "
                                  "every kernel's algorithmic GB/s against P; 12 rounds per point, medians",
-                         "peak_gbs": peak, "peak_kind": peak_kind, "points": run_sweep(peak, frac_key)}
+                         "peak_gbs": peak, "peak_kind": peak_kind, "points": points}
+        if sync:
+            line["sweep"]["sync"] = sync
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         times, what, threads, _ = time_oracle(wl, 1.0 / 2.0, 3)
         base = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": threads,
@@ -652,7 +742,10 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--min-seconds", type=float, default=0.5,
                     help="the K-round timed region is repeated until this much has been timed")
-    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--sweep", default="default", choices=["default", "full", "none"],
+                    help="which set of workloads the sweep against P covers (see sweep_cases)")
+    ap.add_argument("--no-sweep", action="store_true", help="same as --sweep none")
+    ap.add_argument("--table", default="", help="print the markdown tables of a saved JSON line and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-case", action="store_true", help="run the small case for ncu and exit")
     ap.add_argument("--pc-n", type=int, default=8)
@@ -663,6 +756,11 @@ def main():
     ap.add_argument("--pc-reps", type=int, default=2)
     ap.add_argument("--pc-fused", action="store_true", help="hadfl_round instead of the separate calls")
     args = ap.parse_args()
+    if args.no_sweep:
+        args.sweep = "none"
+    if args.table:
+        print_tables(args.table)
+        return
     if args.profile_case:
         run_profile_case(args)
         return

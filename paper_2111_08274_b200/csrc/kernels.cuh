@@ -760,7 +760,17 @@ __device__ __forceinline__ void finish_two_level(const double *__restrict__ part
     double s = 0.0;
     for (int l = lane; l < g_size; l += 32) s += __ldcg(src + l);
     s = warp_sum(s);
-    if (lane == 0 && access_ok(group_partials + (int64_t)t * n_groups + g, 8)) group_partials[(int64_t)t * n_groups + g] = s;
+    if (lane == 0) {
+      if (n_groups == 1) {  // a single group: its sum is the result (the second level would add 0 to it)
+        emit(t, s);
+      } else if (access_ok(group_partials + (int64_t)t * n_groups + g, 8)) {
+        group_partials[(int64_t)t * n_groups + g] = s;
+      }
+    }
+  }
+  if (n_groups == 1) {
+    if (threadIdx.x == 0) group_tickets[g] = 0u;
+    return;
   }
   __threadfence();
   __syncthreads();
