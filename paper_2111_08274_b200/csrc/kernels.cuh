@@ -588,11 +588,10 @@ template <typename WT, int KR, int U>
 __global__ void __launch_bounds__(kThreads)
 k_combine(WT *__restrict__ w, int64_t stride, int64_t n_params, CombineArgs c) {
   constexpr int E = Pack16<WT>::E;
-  // Blocks walk the vector from its END to its start: the kernels before and after this one in a
-  // round (local update, statistics) walk it from the start, so whatever the previous kernel left
-  // in the 126 MB L2 - the end of every row - is read first, and what this kernel leaves there -
-  // the start of the rows it wrote - is what the statistics kernel reads first.  Measured on the
-  // ResNet-18-sized workload inside a round: aggregation 61 -> 57 us, statistics 75 -> 62 us.
+  // Blocks walk the vector from its END to its start: the local update before it in a round walks
+  // it from the start, so what that kernel left in the 126 MB L2 - the end of every row - is read
+  // first.  Measured inside a round on the ResNet-18-sized workload (k = 4): 159 of the 179 MB of
+  // reads come from DRAM instead of all of them, 61 -> 57 us.
   const int64_t chunk = (int64_t)(gridDim.x - 1 - blockIdx.x);
   const int64_t p0 = chunk * (kThreads * U) + threadIdx.x;
   // Fast path (all but the last chunk of a launch): every pack of the block is full, so the
