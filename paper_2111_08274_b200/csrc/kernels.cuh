@@ -21,6 +21,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "debug_check.cuh"
 #include "philox.cuh"
 
@@ -487,51 +489,60 @@ __global__ void __launch_bounds__(kThreads)
 k_local_step(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, LocalStepArgs a,
              PhiloxKeys keys, StepConsts k) {
   const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  const int live = live_of(n_params, p, E);
-  if (live == 0) return;
-  const GroupProducts<E / 4> gp(p);
-  char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
-  char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
+  // The body is compiled twice: for blocks whose packs are all full (`live` is then the constant
+  // E and every ragged-tail test in the loads and stores folds away: 2-3 % fewer instructions per
+  // row) and for the one block that holds the end of the vector.
+  auto run = [&](auto all_full) {
+    const int live = decltype(all_full)::value ? E : live_of(n_params, p, E);
+    if (live == 0) return;
+    const GroupProducts<E / 4> gp(p);
+    char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
+    char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
 
-  auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
-    ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-    ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
-  };
-  auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
-    sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-    if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
-    st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-    st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
-  };
-  // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
-  auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
-    if constexpr (sizeof(WT) == 4) {
-      body(j, rw.v, rm.v);
-    } else if constexpr (sizeof(MT) == 4) {
-      float wv[E];
-      unpack(rw, wv);
-      body(j, wv, rm.v);
-    } else {
-      float wv[E], mv[E];
-      unpack(rw, wv);
-      unpack(rm, mv);
-      body(j, wv, mv);
+    auto load = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
+      ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+      ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
+    };
+    auto body = [&](int j, float (&wv)[E], float (&mv)[E]) {
+      sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+      if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
+      st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+      st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
+    };
+    // fp32 values are updated in the registers they were loaded into; bf16 ones are widened first
+    auto visit = [&](int j, RawPack<WT, E> &rw, RawPack<MT, E> &rm) {
+      if constexpr (sizeof(WT) == 4) {
+        body(j, rw.v, rm.v);
+      } else if constexpr (sizeof(MT) == 4) {
+        float wv[E];
+        unpack(rw, wv);
+        body(j, wv, rm.v);
+      } else {
+        float wv[E], mv[E];
+        unpack(rw, wv);
+        unpack(rm, mv);
+        body(j, wv, mv);
+      }
+    };
+    // No prefetch of the next row: the registers it would take cost a resident block, and four
+    // blocks per SM hide the row loads better than three blocks with a prefetch (measured).
+    // Grid: x = chunks of kThreads packs; y = 1: the block walks over all listed rows (every thread
+    // mixes light and heavy rows, so memory-bound and arithmetic-bound phases overlap), or
+    // y = number of rows: one row per block (eight times more, shorter blocks: no partial last
+    // wave, which is worth 5-7 % when every row is memory-bound).  The host chooses.
+    RawPack<WT, E> rw;
+    RawPack<MT, E> rm;
+    const int j_begin = gridDim.y > 1 ? (int)blockIdx.y : 0;
+    const int j_end = gridDim.y > 1 ? j_begin + 1 : a.n;
+    for (int j = j_begin; j < j_end; ++j) {
+      load(j, rw, rm);
+      visit(j, rw, rm);
     }
   };
-  // No prefetch of the next row: the registers it would take cost a resident block, and four
-  // blocks per SM hide the row loads better than three blocks with a prefetch (measured).
-  // Grid: x = chunks of kThreads packs; y = 1: the block walks over all listed rows (every thread
-  // mixes light and heavy rows, so memory-bound and arithmetic-bound phases overlap), or
-  // y = number of rows: one row per block (eight times more, shorter blocks: no partial last
-  // wave, which is worth 5-7 % when every row is memory-bound).  The host chooses.
-  RawPack<WT, E> rw;
-  RawPack<MT, E> rm;
-  const int j_begin = gridDim.y > 1 ? (int)blockIdx.y : 0;
-  const int j_end = gridDim.y > 1 ? j_begin + 1 : a.n;
-  for (int j = j_begin; j < j_end; ++j) {
-    load(j, rw, rm);
-    visit(j, rw, rm);
-  }
+  if (((int64_t)blockIdx.x + 1) * kThreads * E <= n_params)
+    run(std::true_type{});
+  else
+    run(std::false_type{});
 }
 
 // ------------------------------------------------------------------------------------------
@@ -944,90 +955,99 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
   const int64_t n_packs = (n_params + E - 1) / E;
   const int64_t n_chunks = (n_packs + kThreads - 1) / kThreads;
   for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
-    const int64_t p = chunk * kThreads + threadIdx.x;
-    const int live = live_of(n_params, p, E);
-    const GroupProducts<E / 4> gp(p);
-    char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
-    char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
+    // The chunk's work is compiled twice: for chunks whose packs are all full (`live` is then the
+    // constant E and every ragged-tail test in the loads and stores folds away) and for the chunk
+    // that holds the end of the vector (and, there, the lanes beyond it).
+    auto do_chunk = [&](auto all_full) {
+      const int64_t p = chunk * kThreads + threadIdx.x;
+      const int live = decltype(all_full)::value ? E : live_of(n_params, p, E);
+      const GroupProducts<E / 4> gp(p);
+      char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
+      char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
 
-    // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
-    // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
-    // 0).  fp32 values are updated in the registers they were loaded into.
-    auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
-      RawPack<WT, E> rw;
-      ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-      const bool stepped = a.r[j].steps > 0;
-      if (stepped) {
-        RawPack<MT, E> rm;
-        ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
-        float mv[E];
-        unpack(rw, wv);
-        unpack(rm, mv);
-        sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-        if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
-        st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
-#pragma unroll
-        for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
-        if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
-#pragma unroll
-          for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
+      // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
+      // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
+      // 0).  fp32 values are updated in the registers they were loaded into.
+      auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
+        RawPack<WT, E> rw;
+        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+        const bool stepped = a.r[j].steps > 0;
+        if (stepped) {
+          RawPack<MT, E> rm;
+          ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
+          float mv[E];
+          unpack(rw, wv);
+          unpack(rm, mv);
+          sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+          if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
+          st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
+  #pragma unroll
+          for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
+          if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
+  #pragma unroll
+            for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
+          }
+        } else {
+          unpack(rw, wv);
         }
-      } else {
-        unpack(rw, wv);
-      }
-      return stepped;
-    };
+        return stepped;
+      };
 
-    // ---- the selected devices in draw order: acc = a_0 w_0, then acc = fma(a_j, w_j, acc)
-    float acc[E];
-    {
-      float wv[E];
-      row_after_steps(0, wv);
-      const float a0 = a.a[0];
-#pragma unroll
-      for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
-    }
-    for (int j = 1; j < a.k; ++j) {
-      float wv[E];
-      row_after_steps(j, wv);
-      const float aj = a.a[j];
-#pragma unroll
-      for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
-    }
-    {
-      float n2 = 0.f;
-#pragma unroll
-      for (int i = 0; i < E; ++i) {
-        acc[i] = as_stored(acc[i], w);
-        n2 = fmaf(acc[i], acc[i], n2);
+      // ---- the selected devices in draw order: acc = a_0 w_0, then acc = fma(a_j, w_j, acc)
+      float acc[E];
+      {
+        float wv[E];
+        row_after_steps(0, wv);
+        const float a0 = a.a[0];
+  #pragma unroll
+        for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
       }
-      // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
-      if (a.k > 1 || a.r[0].steps > 0)
-        for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
-      add_row_sums(s_acc, a.k - 1, n2, 0.f, lane);  // one value for all selected devices
-    }
-    // ---- the other devices: keep their own model, or receive the aggregate
-    for (int j = a.k; j < a.n; ++j) {
-      float wv[E];
-      const bool stepped = row_after_steps(j, wv);
-      if (a.write_all == 1) {
-#pragma unroll
-        for (int i = 0; i < E; ++i) wv[i] = acc[i];
-      } else if (a.write_all == 2) {
-#pragma unroll
-        for (int i = 0; i < E; ++i)
-          wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
+      for (int j = 1; j < a.k; ++j) {
+        float wv[E];
+        row_after_steps(j, wv);
+        const float aj = a.a[j];
+  #pragma unroll
+        for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
       }
-      if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-      float n2 = 0.f, d2 = 0.f;
-#pragma unroll
-      for (int i = 0; i < E; ++i) {
-        const float d = wv[i] - acc[i];
-        n2 = fmaf(wv[i], wv[i], n2);
-        d2 = fmaf(d, d, d2);
+      {
+        float n2 = 0.f;
+  #pragma unroll
+        for (int i = 0; i < E; ++i) {
+          acc[i] = as_stored(acc[i], w);
+          n2 = fmaf(acc[i], acc[i], n2);
+        }
+        // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
+        if (a.k > 1 || a.r[0].steps > 0)
+          for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
+        add_row_sums(s_acc, a.k - 1, n2, 0.f, lane);  // one value for all selected devices
       }
-      add_row_sums(s_acc, j, n2, d2, lane);
-    }
+      // ---- the other devices: keep their own model, or receive the aggregate
+      for (int j = a.k; j < a.n; ++j) {
+        float wv[E];
+        const bool stepped = row_after_steps(j, wv);
+        if (a.write_all == 1) {
+  #pragma unroll
+          for (int i = 0; i < E; ++i) wv[i] = acc[i];
+        } else if (a.write_all == 2) {
+  #pragma unroll
+          for (int i = 0; i < E; ++i)
+            wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
+        }
+        if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+        float n2 = 0.f, d2 = 0.f;
+  #pragma unroll
+        for (int i = 0; i < E; ++i) {
+          const float d = wv[i] - acc[i];
+          n2 = fmaf(wv[i], wv[i], n2);
+          d2 = fmaf(d, d, d2);
+        }
+        add_row_sums(s_acc, j, n2, d2, lane);
+      }
+    };
+    if ((chunk + 1) * kThreads * E <= n_params)
+      do_chunk(std::true_type{});
+    else
+      do_chunk(std::false_type{});
   }
   // ---- block: sum the per-thread slots of every visit index j >= k - 1.  Warp w takes the visit
   // indices k - 1 + w, k - 1 + w + 8, ...: each lane adds the slots of the threads that share its
