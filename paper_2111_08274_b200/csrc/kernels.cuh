@@ -981,10 +981,10 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
           sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
           if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
           st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
           if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
-  #pragma unroll
+#pragma unroll
             for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
           }
         } else {
@@ -999,19 +999,19 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
         float wv[E];
         row_after_steps(0, wv);
         const float a0 = a.a[0];
-  #pragma unroll
+#pragma unroll
         for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
       }
       for (int j = 1; j < a.k; ++j) {
         float wv[E];
         row_after_steps(j, wv);
         const float aj = a.a[j];
-  #pragma unroll
+#pragma unroll
         for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
       }
       {
         float n2 = 0.f;
-  #pragma unroll
+#pragma unroll
         for (int i = 0; i < E; ++i) {
           acc[i] = as_stored(acc[i], w);
           n2 = fmaf(acc[i], acc[i], n2);
@@ -1026,16 +1026,16 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
         float wv[E];
         const bool stepped = row_after_steps(j, wv);
         if (a.write_all == 1) {
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < E; ++i) wv[i] = acc[i];
         } else if (a.write_all == 2) {
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < E; ++i)
             wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
         }
         if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
         float n2 = 0.f, d2 = 0.f;
-  #pragma unroll
+#pragma unroll
         for (int i = 0; i < E; ++i) {
           const float d = wv[i] - acc[i];
           n2 = fmaf(wv[i], wv[i], n2);
