@@ -69,8 +69,10 @@ ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to 
 # element-step in fewer cycles than its busiest pipe needs, so
 #   peak = SMs x 4 sub-partitions x SM clock / max(PIPE_CYCLES)      [element-steps per second]
 # with the SM clock sampled during the timed region.  "issue" is the warp scheduler's issue slot
-# (one instruction per cycle); the integer multiplies of Philox occupy the FMA-heavy pipe.
-PIPE_CYCLES_PER_ELEM_STEP = {"fmaheavy": 0.6141, "issue": 0.6046, "xu": 0.5000, "alu": 0.3572, "fmalite": 0.2667}
+# (one instruction per cycle: 154.8 warp instructions per step and 8-parameter pack); "fmaheavy"
+# counts only what no scheduling can move off that pipe, the 36 32x32->64-bit multiplies of Philox
+# at 4 cycles each (with the FP32 instructions the hardware places there it is busy 0.60-0.63).
+PIPE_CYCLES_PER_ELEM_STEP = {"issue": 0.6046, "fmaheavy": 0.5625, "xu": 0.5000, "alu": 0.3652, "fmalite": 0.2511}
 PIPE_CYCLES_SOURCE = "profiles/k_local_step_pipes_N8_P4M.md"
 
 # DRAM bytes per unit of work moved by one launch, from the ncu captures summarised under profiles/
@@ -80,7 +82,7 @@ PIPE_CYCLES_SOURCE = "profiles/k_local_step_pipes_N8_P4M.md"
 # not counted.  Unit: (device, parameter) for the round, the local update and the statistics, one
 # element of a selected row for the aggregation.  None = not captured for the kernel as it stands.
 NCU_DRAM_READ_PER_UNIT = {"round": 8.00, "local_step": 8.00, "aggregate": 4.00, "stats": 4.00}
-NCU_DRAM_WRITE_PER_UNIT = {"round": 6.13, "local_step": 6.12, "aggregate": 0.30, "stats": 0.004}
+NCU_DRAM_WRITE_PER_UNIT = {"round": 6.12, "local_step": 6.12, "aggregate": 0.26, "stats": 0.003}
 NCU_DRAM_SOURCE = "profiles/kernels_small_case_N8_P4M.md"
 
 
