@@ -79,7 +79,8 @@ int for_storage(const hadfl_handle *h, F &&f) {
                     : f(TypeTag<__nv_bfloat16>{}, TypeTag<float>{}, IntTag<0>{});
 }
 
-constexpr int kRowPerBlockMaxSteps = 2;  // local update: one row per block up to this many steps
+constexpr int kRowPerBlockMaxSteps = 2;  // up to this many steps per device a launch is memory-bound: the local update
+                                         // then takes one row per block (fp32), the fused round prefetches rows (bf16)
 constexpr int kStatsU = 4;  // 16-byte packs per thread and chunk in the statistics kernel
 constexpr int64_t kRoundGridCap = 16384;  // most blocks of a fused-round launch (bounds its scratch: 8 MB)
 
@@ -253,9 +254,24 @@ int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
     using WT = typename decltype(wt)::type;
     using MT = typename decltype(mt)::type;
     const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
-    k_round<WT, MT, NormalsFast, StepPack<WT>::E, decltype(rm)::value><<<h->round_grid, kThreads, smem, h->stream>>>(
-        (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-        h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
+    constexpr int E = StepPack<WT>::E;
+    constexpr int RM = decltype(rm)::value;
+    // bf16 parameters and at most two steps per device: the build that prefetches the next row
+    int max_steps = 0;
+    for (int j = 0; j < a.n; ++j) max_steps = a.r[j].steps > max_steps ? a.r[j].steps : max_steps;
+    bool prefetch = false;
+    if constexpr (sizeof(WT) == 2) {
+      if (max_steps <= kRowPerBlockMaxSteps) {
+        prefetch = true;
+        k_round<WT, MT, NormalsFast, E, RM, true><<<h->round_grid, kThreads, smem, h->stream>>>(
+            (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+            h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
+      }
+    }
+    if (!prefetch)
+      k_round<WT, MT, NormalsFast, E, RM, false><<<h->round_grid, kThreads, smem, h->stream>>>(
+          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
+          h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
     return check_launch(h);
   });
 }

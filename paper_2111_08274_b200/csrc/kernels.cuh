@@ -915,6 +915,11 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 // the end of the block, per row, a fixed-order sum over the warps and a butterfly over each
 // half-warp (fp64) -> partials[value][block]; two-level last-ticket finish.  Deterministic.
 // Dynamic shared memory: n * kThreads floats.  64 registers: four resident blocks per SM.
+// PF = true is a second build that issues the next row's loads before the current row's steps
+// (80 registers, three resident blocks).  With bf16 parameters a row is 48 bytes per thread or
+// less, and when every device runs one or two steps the launch is bound by how many bytes are in
+// flight: the prefetch is worth 6-8 % there (and costs 1-3 % with more steps, and 0-13 % with fp32
+// parameters at any step count), so the host takes it for exactly that case.
 // ------------------------------------------------------------------------------------------
 struct RoundArgs {
   int32_t n;          // rows visited = all N devices: [0, k) selected in draw order, then the rest
@@ -940,8 +945,8 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
 
 constexpr int kRoundBlocksPerSM = 4;
 
-template <typename WT, typename MT, typename Gen, int E, int RM>
-__global__ void __launch_bounds__(kThreads, kRoundBlocksPerSM)
+template <typename WT, typename MT, typename Gen, int E, int RM, bool PF>
+__global__ void __launch_bounds__(kThreads, PF ? kRoundBlocksPerSM - 1 : kRoundBlocksPerSM)
 k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
         StepConsts k, double *__restrict__ partials, double *__restrict__ group_partials,
         unsigned int *__restrict__ group_tickets, unsigned int *__restrict__ ticket,
@@ -968,13 +973,27 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
       // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
       // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
       // 0).  fp32 values are updated in the registers they were loaded into.
+      // PF: the next row's loads are issued before this row's steps (see the kernel's header).
+      RawPack<WT, E> rw_next;
+      RawPack<MT, E> rm_next;
+      auto fetch = [&](int j) {
+        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw_next);
+        if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm_next);
+      };
+      if constexpr (PF) fetch(0);
       auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
         RawPack<WT, E> rw;
-        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+        RawPack<MT, E> rm;
+        if constexpr (PF) {
+          rw = rw_next;
+          rm = rm_next;
+          if (j + 1 < a.n) fetch(j + 1);
+        } else {
+          ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
+        }
         const bool stepped = a.r[j].steps > 0;
         if (stepped) {
-          RawPack<MT, E> rm;
-          ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
+          if constexpr (!PF) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
           float mv[E];
           unpack(rw, wv);
           unpack(rm, mv);

@@ -92,6 +92,37 @@ def test_fused_round_with_mixed_global_synchronisation(oracle, n, P, k, beta, dt
     plain.close()
 
 
+@pytest.mark.parametrize("dtype,m_dtype,rounding", [(0, 0, 0), (1, 0, 0), (1, 1, 0), (1, 0, 1), (1, 1, 1)])
+@pytest.mark.parametrize("n,P,k,beta", [(6, 70_003, 2, 1.0), (16, 9_999, 4, 0.5), (3, 300_007, 3, 1.0), (5, 7, 1, 0.25)])
+def test_fused_round_when_no_device_runs_more_than_two_steps(oracle, n, P, k, beta, dtype, m_dtype, rounding):
+    """At most two steps per device is the memory-bound regime, for which the library picks other
+    launch shapes (one row per block in the local update; with bf16 parameters a build of the fused
+    round that loads the next row ahead).  Some devices run no step at all; every second round is a
+    global synchronisation (overwrite or mix).  Fused round against the separate calls bit for bit,
+    selections and versions against the oracle, parameters within the storage's tolerance."""
+    steps = tuple((i * 5 + 1) % 3 for i in range(n))          # 0, 1 and 2 steps
+    wl = wl_of(n, P, k, dtype=dtype, steps=steps, sync_every=2, sync_beta=beta, m_dtype=m_dtype, rounding=rounding)
+    fused, plain = runtime.Arena(wl), runtime.Arena(wl)
+    sim = make_sim(oracle, wl)
+    for r in range(wl.rounds):
+        sf, sp, so = fused.run_round_fused(r), plain.run_round(r), oracle_round(sim, wl, r)
+        assert np.array_equal(sf, sp) and np.array_equal(sf, so), r
+        assert np.array_equal(fused.h.get_versions()[0], sim.get_versions()[0]), r
+        n2, d2 = fused.h.stats_read()
+        pn2, pd2 = plain.h.stats_read()
+        assert np.allclose(n2, pn2, rtol=2e-6) and np.allclose(d2, pd2, rtol=2e-6, atol=1e-30), r
+    assert_same_state(fused, plain, n)
+    for i in range(n):
+        got, want = fused.h.read_params(i), sim.read_params(i)
+        if dtype == 0:
+            assert_close_params(got, want, "w[%d]" % i)
+        else:
+            assert np.abs(got - want).max() <= 2 * bf16_ulp(np.abs(want).max()) and np.mean(got != want) < 0.02
+    fused.h.debug_check()
+    fused.close()
+    plain.close()
+
+
 @pytest.mark.parametrize("dtype", [0, 1])
 def test_a_run_of_rounds_in_one_call_equals_the_rounds_one_by_one(dtype):
     from dataclasses import replace
