@@ -123,10 +123,10 @@ def test_fused_round_when_no_device_runs_more_than_two_steps(oracle, n, P, k, be
     plain.close()
 
 
-@pytest.mark.parametrize("dtype", [0, 1])
-def test_a_run_of_rounds_in_one_call_equals_the_rounds_one_by_one(dtype):
+@pytest.mark.parametrize("dtype,steps_hi", [(0, 8), (1, 8), (1, 2)])
+def test_a_run_of_rounds_in_one_call_equals_the_rounds_one_by_one(dtype, steps_hi):
     from dataclasses import replace
-    wl = replace(workloads.shrink(workloads.c2(), 30_011, rounds=9), dtype=dtype, sync_every=4)
+    wl = replace(workloads.shrink(workloads.c2(), 30_011, rounds=9), dtype=dtype, sync_every=4, steps_hi=steps_hi)
     one, many = runtime.Arena(wl), runtime.Arena(wl)
     want = np.stack([one.run_round_fused(r) for r in range(wl.rounds)])
     got = np.concatenate([many.run_rounds_fused(0, 5), many.run_rounds_fused(5, 4)])
