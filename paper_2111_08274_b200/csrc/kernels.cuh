@@ -247,30 +247,43 @@ __device__ __forceinline__ float r2_next_to_one(uint32_t x0, float scale2) {
 }
 
 struct NormalsFast {
-  // Two normals of standard deviation s from two words; the caller passes lg_scale = -2 ln2 s^2
-  // and scale2 = s^2 so that the scaling costs no instruction:
+  // The four normals of standard deviation s of one Philox block (words x0 .. x3; pairs (x0, x1)
+  // and (x2, x3)); the caller passes lg_scale = -2 ln2 s^2 and scale2 = s^2 so that the scaling
+  // costs no instruction:
   //   r^2 = lg_scale * lg2(u0)            (u0 = (x0 + 0.5) 2^-32)
   //   theta = 2 pi a,  a = ((int)x1 + 0.5) 2^-32          (one fused multiply-add)
+  // The fp32 arithmetic is written on packed pairs (sm_100's two-wide fp32 instructions: one issue
+  // slot, two IEEE results): the block's two radii, its two angles, the two normals of a pair.
   // Next to u0 = 1 (x0 >= 2^32 - 2^22) lg2.approx only has an absolute error bound, so the exact
   // complement and a series take over.  Measured against a double-precision evaluation (s = 1):
   // max |dz| about 2e-6, mean 1.6e-7.
   static constexpr uint32_t kNearOne = 0xFFC00000u;
-  // r^2 away from u0 = 1 (wrong by up to a few 1e-7 absolute next to it: see needs_series)
-  static __device__ __forceinline__ float radius2(uint32_t x0, float lg_scale) {
-    return lg_scale * sfu_lg2(fmaf(__uint2float_rn(x0), 0x1p-32f, 0x1p-33f));
+  // r^2 of both pairs, away from u0 = 1 (wrong by up to a few 1e-7 absolute next to it: see needs_series)
+  static __device__ __forceinline__ float2 radius2_pair(uint32_t x0, uint32_t x2, float lg_scale) {
+    const float2 u = __ffma2_rn(make_float2(__uint2float_rn(x0), __uint2float_rn(x2)),
+                                make_float2(0x1p-32f, 0x1p-32f), make_float2(0x1p-33f, 0x1p-33f));
+    return __fmul2_rn(make_float2(lg_scale, lg_scale), make_float2(sfu_lg2(u.x), sfu_lg2(u.y)));
   }
   static __device__ __forceinline__ bool needs_series(uint32_t x0) { return x0 >= kNearOne; }
-  static __device__ __forceinline__ void finish(float r2, uint32_t x1, float &z0, float &z1) {
-    const float theta = fmaf(__int2float_rn((int)x1), 1.4629180792671596e-9f, 7.314590396335798e-10f);
-    const float r = sfu_sqrt(r2);
-    z0 = r * sfu_cos(theta);
-    z1 = r * sfu_sin(theta);
+  // theta of both pairs (words 1 and 3)
+  static __device__ __forceinline__ float2 angle_pair(uint32_t x1, uint32_t x3) {
+    return __ffma2_rn(make_float2(__int2float_rn((int)x1), __int2float_rn((int)x3)),
+                      make_float2(1.4629180792671596e-9f, 1.4629180792671596e-9f),
+                      make_float2(7.314590396335798e-10f, 7.314590396335798e-10f));
   }
-  static __device__ __forceinline__ void pair(uint32_t x0, uint32_t x1, float lg_scale,
-                                              float scale2, float &z0, float &z1) {
-    float r2 = radius2(x0, lg_scale);
-    if (needs_series(x0)) r2 = r2_next_to_one(x0, scale2);
-    finish(r2, x1, z0, z1);
+  // (r cos theta, r sin theta)
+  static __device__ __forceinline__ float2 finish_pair(float r2, float theta) {
+    const float r = sfu_sqrt(r2);
+    return __fmul2_rn(make_float2(r, r), make_float2(sfu_cos(theta), sfu_sin(theta)));
+  }
+  static __device__ __forceinline__ float4 block(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
+                                                 float lg_scale, float scale2) {
+    float2 r2 = radius2_pair(x0, x2, lg_scale);
+    if (needs_series(x0)) r2.x = r2_next_to_one(x0, scale2);
+    if (needs_series(x2)) r2.y = r2_next_to_one(x2, scale2);
+    const float2 theta = angle_pair(x1, x3);
+    const float2 z01 = finish_pair(r2.x, theta.x), z23 = finish_pair(r2.y, theta.y);
+    return make_float4(z01.x, z01.y, z23.x, z23.y);
   }
 };
 
@@ -295,6 +308,13 @@ struct NormalsAccurate {
     z0 = r * c;
     z1 = r * s;
   }
+  static __device__ __forceinline__ float4 block(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
+                                                 float lg_scale, float scale2) {
+    float4 z;
+    pair(x0, x1, lg_scale, scale2, z.x, z.y);
+    pair(x2, x3, lg_scale, scale2, z.z, z.w);
+    return z;
+  }
 };
 
 constexpr float kMinusTwoLn2 = -1.3862943611198906f;
@@ -304,10 +324,7 @@ template <typename Gen>
 __device__ __forceinline__ float4 normals_of_block(uint32_t c0, uint32_t c1, uint32_t c2,
                                                    uint32_t c3, const PhiloxKeys &keys) {
   philox4x32_10(c0, c1, c2, c3, keys);
-  float4 z;
-  Gen::pair(c0, c1, kMinusTwoLn2, 1.0f, z.x, z.y);
-  Gen::pair(c2, c3, kMinusTwoLn2, 1.0f, z.z, z.w);
-  return z;
+  return Gen::block(c0, c1, c2, c3, kMinusTwoLn2, 1.0f);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -387,10 +404,28 @@ struct GroupProducts {
   }
 };
 
+// One SGD step of two parameters on packed pairs:
+//   g = fma(wd, w, noise);  m = fma(mu, m, g);  w = fma(-lr, m, w)        (per lane, as in Eq. 3)
+__device__ __forceinline__ void sgd_update_pair(float &w0, float &w1, float &m0, float &m1, float2 noise,
+                                                float2 wd2, float2 mu2, float2 neg_lr2) {
+  const float2 w2 = make_float2(w0, w1);
+  const float2 g2 = __ffma2_rn(wd2, w2, noise);
+  const float2 m2 = __ffma2_rn(mu2, make_float2(m0, m1), g2);
+  const float2 w2n = __ffma2_rn(neg_lr2, m2, w2);
+  w0 = w2n.x; w1 = w2n.y;
+  m0 = m2.x; m1 = m2.y;
+}
+
 // The steps of one device on one pack.  Each step is written stage by stage over all NB Philox
 // blocks of the pack - all generator rounds, then all radii, one combined test for the rare
 // "u0 next to 1" case, then all angles, then the update - so that the independent chains sit in
 // the same straight-line code and the hardware scheduler can interleave them.
+// The fp32 arithmetic of a step is written on pairs (sm_100's two-wide fp32 instructions: one
+// issue slot, two IEEE results, so every value is bit for bit what the scalar form gives): the two
+// radii of a block, its two angles, the two normals of a Box-Muller pair and their two parameters.
+// The launch is bound by the issue slot with several steps per device, and this takes 22 of 155
+// warp instructions out of a step of an 8-parameter pack (measured: K1 -3 ... -4 %, fused round
+// -4 ... -5 %).
 template <typename Gen, int NB>
 __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB],
                                           const GroupProducts<NB> &gp, const RowStep &rs,
@@ -398,6 +433,8 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
   uint32_t c2_first[NB];
 #pragma unroll
   for (int b = 0; b < NB; ++b) c2_first[b] = gp.hi[b] ^ rs.r1_c2;
+  const float2 wd2 = make_float2(k.wd, k.wd), mu2 = make_float2(k.mu, k.mu);
+  const float2 neg_lr2 = make_float2(k.neg_lr, k.neg_lr);
   for (int e = 0; e < rs.steps; ++e) {
     const uint32_t c0_first = rs.r1_c0 ^ (rs.base_lo + (uint32_t)e);
     uint32_t x[NB][4];
@@ -409,32 +446,27 @@ __device__ __forceinline__ void sgd_steps(float (&w)[4 * NB], float (&m)[4 * NB]
     for (int r = 1; r < 10; ++r)
 #pragma unroll
       for (int b = 0; b < NB; ++b) philox_round(x[b][0], x[b][1], x[b][2], x[b][3], keys.a[r], keys.b[r]);
-    float r2[NB][2];
+    float2 r2[NB];  // squared radii of the block's two pairs
     uint32_t top = 0;
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      r2[b][0] = Gen::radius2(x[b][0], k.lg_scale);
-      r2[b][1] = Gen::radius2(x[b][2], k.lg_scale);
+      r2[b] = Gen::radius2_pair(x[b][0], x[b][2], k.lg_scale);
       top = max(top, max(x[b][0], x[b][2]));
     }
     if (Gen::needs_series(top)) {  // about once in 250 steps of a pack
 #pragma unroll
       for (int b = 0; b < NB; ++b) {
-        if (Gen::needs_series(x[b][0])) r2[b][0] = r2_next_to_one(x[b][0], k.scale2);
-        if (Gen::needs_series(x[b][2])) r2[b][1] = r2_next_to_one(x[b][2], k.scale2);
+        if (Gen::needs_series(x[b][0])) r2[b].x = r2_next_to_one(x[b][0], k.scale2);
+        if (Gen::needs_series(x[b][2])) r2[b].y = r2_next_to_one(x[b][2], k.scale2);
       }
     }
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
-      float n[4];  // grad_std * z
-      Gen::finish(r2[b][0], x[b][1], n[0], n[1]);
-      Gen::finish(r2[b][1], x[b][3], n[2], n[3]);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float g = fmaf(k.wd, w[4 * b + i], n[i]);
-        m[4 * b + i] = fmaf(k.mu, m[4 * b + i], g);
-        w[4 * b + i] = fmaf(k.neg_lr, m[4 * b + i], w[4 * b + i]);
-      }
+      const float2 theta = Gen::angle_pair(x[b][1], x[b][3]);
+      const float2 n01 = Gen::finish_pair(r2[b].x, theta.x);  // grad_std * (z0, z1)
+      const float2 n23 = Gen::finish_pair(r2[b].y, theta.y);  // grad_std * (z2, z3)
+      sgd_update_pair(w[4 * b], w[4 * b + 1], m[4 * b], m[4 * b + 1], n01, wd2, mu2, neg_lr2);
+      sgd_update_pair(w[4 * b + 2], w[4 * b + 3], m[4 * b + 2], m[4 * b + 3], n23, wd2, mu2, neg_lr2);
     }
   }
 }
