@@ -68,11 +68,12 @@ ORACLE_NS_PER_ELEM_STEP = 45e-9   # rough cost of the CPU checker, used only to 
 # command under profiles/k_local_step_pipes_N8_P4M.md).  A sub-partition cannot process an
 # element-step in fewer cycles than its busiest pipe needs, so
 #   peak = SMs x 4 sub-partitions x SM clock / max(PIPE_CYCLES)      [element-steps per second]
-# with the SM clock sampled during the timed region.  "issue" is the warp scheduler's issue slot
-# (one instruction per cycle: 154.8 warp instructions per step and 8-parameter pack); "fmaheavy"
-# counts only what no scheduling can move off that pipe, the 36 32x32->64-bit multiplies of Philox
-# at 4 cycles each (with the FP32 instructions the hardware places there it is busy 0.60-0.63).
-PIPE_CYCLES_PER_ELEM_STEP = {"issue": 0.6046, "fmaheavy": 0.5625, "xu": 0.5000, "alu": 0.3652, "fmalite": 0.2511}
+# with the SM clock sampled during the timed region.  "fmaheavy" counts only what no scheduling can
+# move off that pipe, the 36 32x32->64-bit multiplies of Philox per step and 8-parameter pack at 4
+# cycles each (with the packed FP32 instructions the hardware runs there it is busy 0.69); "issue"
+# is the warp scheduler's issue slot (one instruction per cycle: 132.8 warp instructions per step
+# and pack).
+PIPE_CYCLES_PER_ELEM_STEP = {"fmaheavy": 0.5625, "issue": 0.5186, "xu": 0.5000, "alu": 0.3572, "fmalite": 0.1925}
 PIPE_CYCLES_SOURCE = "profiles/k_local_step_pipes_N8_P4M.md"
 
 # DRAM bytes per unit of work moved by one launch, from the ncu captures summarised under profiles/
