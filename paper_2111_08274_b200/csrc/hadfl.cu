@@ -162,12 +162,12 @@ int debug_error(uint64_t *addr) {
   if (addr) *addr = now.bad_addr;
   return now.error ? 1 : 0;
 }
-#define HADFL_DEBUG_VERDICT()                            \
+#define HADFL_DEBUG_RESULT()                            \
   do {                                                   \
     if (debug_error(nullptr)) return HADFL_ERR_STATE;    \
   } while (0)
 #else
-#define HADFL_DEBUG_VERDICT() \
+#define HADFL_DEBUG_RESULT() \
   do {                        \
   } while (0)
 #endif
@@ -314,7 +314,7 @@ int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool moment
   DeviceGuard guard(h->device);
   if (count == 0) {
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
-    HADFL_DEBUG_VERDICT();
+    HADFL_DEBUG_RESULT();
     return HADFL_OK;
   }
   const void *arena = momentum ? h->m : h->w;
@@ -323,14 +323,14 @@ int read_row(hadfl_handle *h, int32_t id, float *dst, int64_t count, bool moment
     HADFL_CUDA(h, cudaMemcpyAsync(dst, src, sizeof(float) * (size_t)count, cudaMemcpyDeviceToHost,
                                   h->stream));
     HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
-    HADFL_DEBUG_VERDICT();
+    HADFL_DEBUG_RESULT();
     return HADFL_OK;
   }
   std::vector<uint16_t> tmp((size_t)count);
   const uint16_t *src = (const uint16_t *)arena + (int64_t)id * h->stride;
   HADFL_CUDA(h, cudaMemcpyAsync(tmp.data(), src, 2 * (size_t)count, cudaMemcpyDeviceToHost, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
-  HADFL_DEBUG_VERDICT();
+  HADFL_DEBUG_RESULT();
   for (int64_t p = 0; p < count; ++p) {
     const uint32_t bits = (uint32_t)tmp[(size_t)p] << 16;
     memcpy(dst + p, &bits, 4);
@@ -774,7 +774,7 @@ int hadfl_stats_read(hadfl_handle *h, float *out_norm2, float *out_div2) {
   HADFL_CUDA(h, cudaMemcpyAsync(buf, h->d_stats, sizeof(float) * 2 * (size_t)n,
                                 cudaMemcpyDeviceToHost, h->stream));
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
-  HADFL_DEBUG_VERDICT();
+  HADFL_DEBUG_RESULT();
   memcpy(out_norm2, buf, sizeof(float) * (size_t)n);
   memcpy(out_div2, buf + n, sizeof(float) * (size_t)n);
   return HADFL_OK;
@@ -974,7 +974,7 @@ int hadfl_synchronize(hadfl_handle *h) {
   if (!h) return HADFL_ERR_INVALID;
   DeviceGuard guard(h->device);
   HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
-  HADFL_DEBUG_VERDICT();
+  HADFL_DEBUG_RESULT();
   return HADFL_OK;
 }
 
