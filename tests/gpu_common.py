@@ -60,10 +60,10 @@ def compare_sample(arena, sim, groups, what):
     return worst
 
 
-def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=(), fused=False):
+def run_and_compare(oracle, wl, groups, check_rounds, stats_rounds=(), fused=False, openmp=False):
     from paper_2111_08274_b200 import runtime
     arena = runtime.Arena(wl)
-    sim = make_sim(oracle, wl, groups)
+    sim = make_sim(oracle, wl, groups, openmp=openmp)
     full = groups is None
     g = np.arange((wl.n_params + 3) // 4, dtype=np.uint32) if full else groups
     worst = 0.0

@@ -15,8 +15,11 @@ def oracle_round(sim, wl, r):
     return sel
 
 
-def make_sim(oracle, wl, groups=None):
+def make_sim(oracle, wl, groups=None, openmp=False):
+    """openmp=True: the oracle's -fopenmp build (same source, same results bit for bit -
+    tests/test_oracle_openmp.py -, its column loops split over the host cores), for column samples
+    too large for one core to follow in seconds."""
     return oracle.Sim(wl.n_devices, wl.n_params, dtype=wl.dtype, momentum=wl.momentum,
                       weight_decay=wl.weight_decay, grad_std=wl.grad_std, init_std=wl.init_std,
                       seed=wl.seed, version_scale=wl.version_scale, weight_mode=wl.weight_mode,
-                      groups=groups, m_dtype=wl.m_dtype, rounding=wl.rounding)
+                      groups=groups, m_dtype=wl.m_dtype, rounding=wl.rounding, openmp=openmp)

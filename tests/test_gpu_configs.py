@@ -50,8 +50,20 @@ def test_c2_full_size_fused_round_sampled_columns(oracle):
     """The launch configuration the benchmark times: the whole round of the full-size workload in
     one hadfl_round call per round."""
     wl = workloads.c2()
-    groups = workloads.sample_groups(wl.n_params, 65_536, 1024, seed=22, around=seams(wl))   # 2^18 random columns
-    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24), fused=True)
+    # 2^20 random columns (2^18 groups) + the first and last 4096 columns of every row + the seams;
+    # the oracle follows them on all host cores (its -fopenmp build: identical results)
+    groups = workloads.sample_groups(wl.n_params, 262_144, 1024, seed=22, around=seams(wl))
+    run_and_compare(oracle, wl, groups, check_rounds=(0, 9, 24), fused=True, openmp=True)
+
+
+@pytest.mark.parametrize("name,rounds", [("c2", 8), ("c3", 11)])
+def test_full_size_fused_round_whole_arena_against_the_oracle(oracle, name, rounds):
+    """Every parameter and every momentum value of the full-size workload against the oracle (all
+    host cores: its -fopenmp build, identical results), through the fused round, for the first
+    rounds (c3: up to and including its first global synchronisation)."""
+    from dataclasses import replace
+    wl = replace(workloads.by_name(name), rounds=rounds)
+    run_and_compare(oracle, wl, None, check_rounds=(0, rounds - 1), stats_rounds=(0,), fused=True, openmp=True)
 
 
 def test_c3_full_size_fused_round_sampled_columns(oracle):
