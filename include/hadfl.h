@@ -210,6 +210,25 @@ int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps
 int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const int32_t *steps, float lr,
                  uint64_t seed, int32_t k, int32_t sync_every, int32_t *out_selected);
 
+/* Rounds per launch.  Every operation of a round (Eq. 3, Eq. 5, the send to the other devices) is
+ * elementwise in the parameter index, and the selections (Eq. 8) depend on versions the host knows
+ * beforehand, so hadfl_rounds may hand several consecutive rounds to ONE launch of the fused kernel:
+ * a block takes its columns through all of them before it moves to the next columns, and from the
+ * second round on the replicas are read from L2 instead of HBM.  Results - parameters, momentum,
+ * counters, selections, every round's statistics - are those of the rounds launched one by one,
+ * bit for bit.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
+ * steps, or the whole arena is at most 64 MiB) and launches the others singly.
+ * hadfl_set_round_batch: the most rounds per launch, 1 .. 8 (default 8; 1 = never batch);
+ * HADFL_ERR_INVALID outside that range.  hadfl_round_batch returns the setting (0 for NULL). */
+int hadfl_set_round_batch(hadfl_handle *h, int32_t max_rounds);
+int32_t hadfl_round_batch(const hadfl_handle *h);
+
+/* The statistics that the fused kernel left for the round `back` rounds before the last one of its
+ * most recent launch (back = 0: the last round, the same as hadfl_stats_read).  A launch keeps the
+ * statistics of each of its rounds; HADFL_ERR_STATE when `back` reaches beyond the rounds of that
+ * launch or no fused round has run.  Synchronises the stream. */
+int hadfl_stats_read_round(hadfl_handle *h, int32_t back, float *out_norm2, float *out_div2);
+
 /* Per-replica statistics (not in the paper; diagnostics of how far the replicas have drifted):
  * out_norm2[i] = sum_p w_i[p]^2, out_div2[i] = sum_p (w_i[p] - w_ref[p])^2, N floats each.
  * Deterministic: fixed grid, fixed summation order, fp32 within a chunk, fp64 above.

@@ -95,6 +95,9 @@ SIGNATURES = {
     "hadfl_launch_count": (C.c_uint64, [_H]),
     "hadfl_row_stride": (C.c_int64, [_H]),
     "hadfl_round_grid": (C.c_int32, [_H]),
+    "hadfl_set_round_batch": (C.c_int, [_H, C.c_int32]),
+    "hadfl_round_batch": (C.c_int32, [_H]),
+    "hadfl_stats_read_round": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
     "hadfl_selection_probs": (C.c_int, [_f64p, _u8p, C.c_int32, _f64p]),
     "hadfl_selection_draw": (C.c_int, [_f64p, _u8p, C.c_int32, C.c_int64, C.c_uint64, C.c_int32, _i32p]),
     "hadfl_predict_version": (C.c_int, [_f64p, C.c_int32, C.c_double, C.c_double, _f64p]),
@@ -315,6 +318,14 @@ class Hadfl:
                     "hadfl_stats_read")
         return n2, d2
 
+    def stats_read_round(self, back):
+        """Statistics of the round `back` rounds before the last one of the most recent fused launch."""
+        n2 = np.empty(self.n_devices, dtype=np.float32)
+        d2 = np.empty(self.n_devices, dtype=np.float32)
+        self._check(self._lib.hadfl_stats_read_round(self._h, back, _p(n2, C.c_float), _p(d2, C.c_float)),
+                    "hadfl_stats_read_round")
+        return n2, d2
+
     def stats(self, ref_device):
         n2 = np.empty(self.n_devices, dtype=np.float32)
         d2 = np.empty(self.n_devices, dtype=np.float32)
@@ -395,6 +406,12 @@ class Hadfl:
 
     def round_grid(self):
         return int(self._lib.hadfl_round_grid(self._h))
+
+    def set_round_batch(self, max_rounds):
+        self._check(self._lib.hadfl_set_round_batch(self._h, max_rounds), "hadfl_set_round_batch")
+
+    def round_batch(self):
+        return int(self._lib.hadfl_round_batch(self._h))
 
     def debug_philox(self, counters, key):
         c = _arr(counters, np.uint32).reshape(-1, 4)

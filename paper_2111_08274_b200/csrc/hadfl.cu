@@ -36,10 +36,13 @@ struct hadfl_handle {
   int stats_lanes = 0;  // blocks per row of the statistics kernel
   bool stats_valid = false;
   // fused round kernel scratch
-  double *d_round_partials = nullptr;        // [2 * kMaxDevices][round_grid]
-  double *d_round_group_partials = nullptr;  // [2 * kMaxDevices][groups of kFinishGroup blocks]
-  unsigned int *d_round_ticket = nullptr;    // [0]: the launch's ticket, [1 ...]: one per group
+  double *d_round_partials = nullptr;        // [round of a batch][2 N][round_grid]
+  double *d_round_group_partials = nullptr;  // [round of a batch][2 N][groups of kFinishGroup blocks]
+  unsigned int *d_round_ticket = nullptr;    // [round of a batch][1 + groups]: the round's ticket, one per group
+  float *d_round_stats = nullptr;            // [round of a batch][2 * kMaxDevices]
   int round_grid = 0;
+  int round_batch = kRoundBatchMax;  // most rounds that hadfl_rounds puts into one launch (1: never batch)
+  int last_launch_rounds = 0;        // rounds in the most recent launch of the fused round kernel
   // model backup that overlaps with later rounds: staging row + copy stream
   void *d_backup = nullptr;
   cudaStream_t backup_stream = nullptr;
@@ -249,29 +252,32 @@ int launch_local_step(hadfl_handle *h, const LocalStepArgs &a, float lr) {
   });
 }
 
-int launch_round(hadfl_handle *h, const RoundArgs &a, float lr) {
+template <int NR>
+int launch_round(hadfl_handle *h, const RoundBatch<NR> &b, float lr) {
   return for_storage(h, [&](auto wt, auto mt, auto rm) {
     using WT = typename decltype(wt)::type;
     using MT = typename decltype(mt)::type;
-    const size_t smem = sizeof(float) * kThreads * (size_t)a.n;
+    const size_t smem = sizeof(float) * kThreads * (size_t)h->cfg.n_devices;
     constexpr int E = StepPack<WT>::E;
     constexpr int RM = decltype(rm)::value;
+    const RoundScratch scratch{h->d_round_partials, h->d_round_group_partials, h->d_round_ticket,
+                               h->d_round_stats, h->d_stats};
     // bf16 parameters and at most two steps per device: the build that prefetches the next row
     int max_steps = 0;
-    for (int j = 0; j < a.n; ++j) max_steps = a.r[j].steps > max_steps ? a.r[j].steps : max_steps;
+    for (int r = 0; r < b.n_rounds; ++r)
+      for (int j = 0; j < b.round[r].n; ++j)
+        max_steps = b.round[r].r[j].steps > max_steps ? b.round[r].r[j].steps : max_steps;
     bool prefetch = false;
     if constexpr (sizeof(WT) == 2) {
       if (max_steps <= kRowPerBlockMaxSteps) {
         prefetch = true;
-        k_round<WT, MT, NormalsFast, E, RM, true><<<h->round_grid, kThreads, smem, h->stream>>>(
-            (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-            h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
+        k_round<WT, MT, NormalsFast, E, RM, true, NR><<<h->round_grid, kThreads, smem, h->stream>>>(
+            (WT *)h->w, (MT *)h->m, h->cfg.n_params, b, h->keys, step_consts(h, lr), scratch);
       }
     }
     if (!prefetch)
-      k_round<WT, MT, NormalsFast, E, RM, false><<<h->round_grid, kThreads, smem, h->stream>>>(
-          (WT *)h->w, (MT *)h->m, h->cfg.n_params, a, h->keys, step_consts(h, lr), h->d_round_partials,
-          h->d_round_group_partials, h->d_round_ticket + 1, h->d_round_ticket, h->d_stats);
+      k_round<WT, MT, NormalsFast, E, RM, false, NR><<<h->round_grid, kThreads, smem, h->stream>>>(
+          (WT *)h->w, (MT *)h->m, h->cfg.n_params, b, h->keys, step_consts(h, lr), scratch);
     return check_launch(h);
   });
 }
@@ -436,11 +442,14 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
     h->round_grid = (int)(need < kRoundGridCap ? need : kRoundGridCap);
   }
   const size_t n_groups = (size_t)((h->round_grid + kFinishGroup - 1) / kFinishGroup);
-  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_partials,
-                           sizeof(double) * 2 * kMaxDevices * (size_t)h->round_grid));
-  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_group_partials, sizeof(double) * 2 * kMaxDevices * n_groups));
-  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_ticket, sizeof(unsigned int) * (1 + n_groups)));
-  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int) * (1 + n_groups), h->stream));
+  const size_t round_vals = (size_t)kRoundBatchMax * 2 * (size_t)cfg->n_devices;
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_partials, sizeof(double) * round_vals * (size_t)h->round_grid));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_group_partials, sizeof(double) * round_vals * n_groups));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_ticket, sizeof(unsigned int) * kRoundBatchMax * (1 + n_groups)));
+  HADFL_CUDA(h, cudaMalloc((void **)&h->d_round_stats, sizeof(float) * kRoundBatchMax * 2 * kMaxDevices));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_ticket, 0, sizeof(unsigned int) * kRoundBatchMax * (1 + n_groups),
+                                h->stream));
+  HADFL_CUDA(h, cudaMemsetAsync(h->d_round_stats, 0, sizeof(float) * kRoundBatchMax * 2 * kMaxDevices, h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_ticket, 0, sizeof(unsigned int), h->stream));
   HADFL_CUDA(h, cudaMemsetAsync(h->d_stats, 0, sizeof(float) * 2 * kMaxDevices, h->stream));
 #ifdef HADFL_DEBUG
@@ -448,8 +457,9 @@ int hadfl_init(const hadfl_config *cfg, hadfl_handle **out) {
   debug_add(h->m, elems * m_elem_size(h));
   debug_add(h->d_partials, sizeof(double) * 2 * (size_t)cfg->n_devices * (size_t)lanes);
   debug_add(h->d_stats, sizeof(float) * 2 * kMaxDevices);
-  debug_add(h->d_round_partials, sizeof(double) * 2 * kMaxDevices * (size_t)h->round_grid);
-  debug_add(h->d_round_group_partials, sizeof(double) * 2 * kMaxDevices * n_groups);
+  debug_add(h->d_round_partials, sizeof(double) * round_vals * (size_t)h->round_grid);
+  debug_add(h->d_round_group_partials, sizeof(double) * round_vals * n_groups);
+  debug_add(h->d_round_stats, sizeof(float) * kRoundBatchMax * 2 * kMaxDevices);
   HADFL_CUDA(h, cudaDeviceSynchronize());
   if (debug_publish()) return HADFL_ERR_CUDA;
 #endif
@@ -469,6 +479,7 @@ int hadfl_destroy(hadfl_handle *h) {
   debug_remove(h->d_stats);
   debug_remove(h->d_round_partials);
   debug_remove(h->d_round_group_partials);
+  debug_remove(h->d_round_stats);
   debug_publish();
 #endif
   if (h->own_arena) {
@@ -481,6 +492,7 @@ int hadfl_destroy(hadfl_handle *h) {
   cudaFree(h->d_round_partials);
   cudaFree(h->d_round_group_partials);
   cudaFree(h->d_round_ticket);
+  cudaFree(h->d_round_stats);
   if (h->backup_stream) cudaStreamSynchronize(h->backup_stream);
   cudaFree(h->d_backup);
   if (h->backup_ready) cudaEventDestroy(h->backup_ready);
@@ -658,84 +670,136 @@ int hadfl_set_sync_beta(hadfl_handle *h, float beta) {
   return HADFL_OK;
 }
 
-int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
-                int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
-                int32_t *out_selected) {
-  if (!h || !out_selected) return HADFL_ERR_INVALID;
+namespace {
+
+// One round as the host plans it before anything is enqueued: the steps per row, the selection
+// (which sees the versions as they will be after the local steps) and the kernel's arguments.
+struct RoundPlan {
+  int row_steps[kMaxDevices];
+  int32_t sel[kMaxDevices];
+  bool crosses;  // a step counter crosses a multiple of 2^32 in this round
+  RoundArgs a;
+};
+
+int plan_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, int64_t round,
+               const double *versions, uint64_t seed, int32_t k, int32_t sync_all, RoundPlan &pl) {
   if (!steps || !distinct_ids(h, device_ids, n)) return HADFL_ERR_INVALID;
   const int N = h->cfg.n_devices;
-  int row_steps[kMaxDevices];
-  for (int i = 0; i < N; ++i) row_steps[i] = 0;
-  bool crosses = false;
+  for (int i = 0; i < N; ++i) pl.row_steps[i] = 0;
+  pl.crosses = false;
   for (int j = 0; j < n; ++j) {
     if (steps[j] < 0) return HADFL_ERR_INVALID;
     const uint64_t base = h->step_count[device_ids[j]];
     if ((base + (uint64_t)steps[j]) >> 56) return HADFL_ERR_STATE;
-    if ((base & 0xFFFFFFFFull) + (uint64_t)steps[j] > ((uint64_t)1 << 32)) crosses = true;
-    row_steps[device_ids[j]] = steps[j];
+    if ((base & 0xFFFFFFFFull) + (uint64_t)steps[j] > ((uint64_t)1 << 32)) pl.crosses = true;
+    pl.row_steps[device_ids[j]] = steps[j];
   }
-  // Selection sees the versions as they will be after the local steps.
   double x[kMaxDevices];
   for (int i = 0; i < N; ++i)
-    x[i] = (versions ? versions[i] : (double)(h->version[i] + (uint32_t)row_steps[i])) *
+    x[i] = (versions ? versions[i] : (double)(h->version[i] + (uint32_t)pl.row_steps[i])) *
            h->cfg.version_scale;
-  int32_t sel[kMaxDevices];
-  if (!selection_draw(x, h->avail, N, round, seed, k, sel)) return HADFL_ERR_INVALID;
+  if (!selection_draw(x, h->avail, N, round, seed, k, pl.sel)) return HADFL_ERR_INVALID;
+  if (pl.crosses) return HADFL_OK;
 
-  if (crosses) {
-    // A step counter crosses a multiple of 2^32 in this call (once in 4 billion steps): take the
-    // separate kernels, which split the launch.
-    int rc = hadfl_local_step(h, device_ids, steps, n, lr);
-    if (rc == HADFL_OK) rc = hadfl_aggregate(h, sel, k, versions);
-    if (rc == HADFL_OK && sync_all) {
-      int32_t others[kMaxDevices];
-      int n_others = 0;
-      uint32_t in_sel = 0;
-      for (int j = 0; j < k; ++j) in_sel |= 1u << sel[j];
-      for (int i = 0; i < N; ++i)
-        if (!(in_sel & (1u << i))) others[n_others++] = i;
-      rc = h->sync_beta == 1.0f ? hadfl_broadcast(h, sel[0], others, n_others)
-                                : hadfl_integrate(h, sel[0], others, n_others, h->sync_beta);
-    }
-    if (rc == HADFL_OK) rc = hadfl_stats_enqueue(h, sel[0]);
-    if (rc != HADFL_OK) return rc;
-    for (int j = 0; j < k; ++j) out_selected[j] = sel[j];
-    return HADFL_OK;
-  }
-
-  RoundArgs a;
+  RoundArgs &a = pl.a;
   memset(&a, 0, sizeof(a));
   a.n = N;
   a.k = k;
   a.write_all = sync_all ? (h->sync_beta == 1.0f ? 1 : 2) : 0;
   a.beta = h->sync_beta;
   a.one_minus_beta = 1.0f - h->sync_beta;
-  aggregation_weights(h->cfg.weight_mode, x, h->avail, N, sel, k, a.a);
+  aggregation_weights(h->cfg.weight_mode, x, h->avail, N, pl.sel, k, a.a);
   uint32_t in_sel = 0;
   int pos = 0;
   for (int j = 0; j < k; ++j) {
-    a.r[pos++] = row_step(h, sel[j], h->step_count[sel[j]], row_steps[sel[j]]);
-    in_sel |= 1u << sel[j];
+    a.r[pos++] = row_step(h, pl.sel[j], h->step_count[pl.sel[j]], pl.row_steps[pl.sel[j]]);
+    in_sel |= 1u << pl.sel[j];
   }
   for (int i = 0; i < N; ++i)
-    if (!(in_sel & (1u << i))) a.r[pos++] = row_step(h, i, h->step_count[i], row_steps[i]);
-  {
-    DeviceGuard guard(h->device);
-    const int rc = launch_round(h, a, lr);
-    if (rc != HADFL_OK) return rc;
-  }
+    if (!(in_sel & (1u << i))) a.r[pos++] = row_step(h, i, h->step_count[i], pl.row_steps[i]);
+  return HADFL_OK;
+}
+
+// The host's mirror of the counters after a planned round (fused path).
+void commit_round(hadfl_handle *h, const RoundPlan &pl, int32_t k, int32_t sync_all) {
+  const int N = h->cfg.n_devices;
   for (int i = 0; i < N; ++i) {
-    h->step_count[i] += (uint64_t)row_steps[i];
-    h->version[i] += (uint32_t)row_steps[i];
+    h->step_count[i] += (uint64_t)pl.row_steps[i];
+    h->version[i] += (uint32_t)pl.row_steps[i];
   }
   uint32_t vmax = 0;
-  for (int j = 0; j < k; ++j) vmax = h->version[sel[j]] > vmax ? h->version[sel[j]] : vmax;
-  for (int j = 0; j < k; ++j) h->version[sel[j]] = vmax;
+  for (int j = 0; j < k; ++j) vmax = h->version[pl.sel[j]] > vmax ? h->version[pl.sel[j]] : vmax;
+  for (int j = 0; j < k; ++j) h->version[pl.sel[j]] = vmax;
   if (sync_all)
     for (int i = 0; i < N; ++i)
       if (h->sync_beta == 1.0f || vmax > h->version[i]) h->version[i] = vmax;
-  h->stats_valid = true;
-  for (int j = 0; j < k; ++j) out_selected[j] = sel[j];
+}
+
+// A round whose step counters cross a multiple of 2^32 (once in 4 billion steps): the separate
+// kernels, which split the launch.
+int round_by_separate_calls(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n,
+                            float lr, const double *versions, int32_t k, int32_t sync_all,
+                            const int32_t *sel) {
+  const int N = h->cfg.n_devices;
+  int rc = hadfl_local_step(h, device_ids, steps, n, lr);
+  if (rc == HADFL_OK) rc = hadfl_aggregate(h, sel, k, versions);
+  if (rc == HADFL_OK && sync_all) {
+    int32_t others[kMaxDevices];
+    int n_others = 0;
+    uint32_t in_sel = 0;
+    for (int j = 0; j < k; ++j) in_sel |= 1u << sel[j];
+    for (int i = 0; i < N; ++i)
+      if (!(in_sel & (1u << i))) others[n_others++] = i;
+    rc = h->sync_beta == 1.0f ? hadfl_broadcast(h, sel[0], others, n_others)
+                              : hadfl_integrate(h, sel[0], others, n_others, h->sync_beta);
+  }
+  if (rc == HADFL_OK) rc = hadfl_stats_enqueue(h, sel[0]);
+  if (rc == HADFL_OK) h->last_launch_rounds = 0;
+  return rc;
+}
+
+// Whether hadfl_rounds may put a planned round into a launch together with its neighbours.  A
+// batch pays where a round is bound by memory or by the launch itself: every device runs at most
+// kRowPerBlockMaxSteps steps, or the arena is small against the L2.  With more steps per device
+// the rounds are bound by arithmetic and the batch's indexed arguments cost what L2 saves
+// (measured: 0 ... -3 %), so those rounds are launched one by one.
+constexpr size_t kBatchSmallArenaBytes = (size_t)64 << 20;
+
+bool batchable(const hadfl_handle *h, const RoundPlan &pl) {
+  if (h->round_batch <= 1) return false;
+  const size_t arena = (size_t)h->cfg.n_devices * (size_t)h->cfg.n_params * (elem_size(h) + m_elem_size(h));
+  if (arena <= kBatchSmallArenaBytes) return true;
+  for (int i = 0; i < h->cfg.n_devices; ++i)
+    if (pl.row_steps[i] > kRowPerBlockMaxSteps) return false;
+  return true;
+}
+
+}  // namespace
+
+int hadfl_round(hadfl_handle *h, const int32_t *device_ids, const int32_t *steps, int32_t n, float lr,
+                int64_t round, const double *versions, uint64_t seed, int32_t k, int32_t sync_all,
+                int32_t *out_selected) {
+  if (!h || !out_selected) return HADFL_ERR_INVALID;
+  RoundPlan pl;
+  int rc = plan_round(h, device_ids, steps, n, round, versions, seed, k, sync_all, pl);
+  if (rc != HADFL_OK) return rc;
+  if (pl.crosses) {
+    rc = round_by_separate_calls(h, device_ids, steps, n, lr, versions, k, sync_all, pl.sel);
+    if (rc != HADFL_OK) return rc;
+  } else {
+    RoundBatch<1> b;
+    b.n_rounds = 1;
+    b.round[0] = pl.a;
+    {
+      DeviceGuard guard(h->device);
+      rc = launch_round(h, b, lr);
+      if (rc != HADFL_OK) return rc;
+    }
+    commit_round(h, pl, k, sync_all);
+    h->stats_valid = true;
+    h->last_launch_rounds = 1;
+  }
+  for (int j = 0; j < k; ++j) out_selected[j] = pl.sel[j];
   return HADFL_OK;
 }
 
@@ -743,16 +807,92 @@ int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const i
                  uint64_t seed, int32_t k, int32_t sync_every, int32_t *out_selected) {
   if (!h || !steps || n_rounds < 0 || sync_every < 0) return HADFL_ERR_INVALID;
   const int N = h->cfg.n_devices;
-  int32_t ids[kMaxDevices], sel[kMaxDevices];
+  int32_t ids[kMaxDevices];
   for (int i = 0; i < N; ++i) ids[i] = i;
+  // Rounds are planned on the host one after the other (each sees the counters the previous one
+  // leaves).  Rounds that gain from it are collected into batches of up to round_batch rounds per
+  // launch; the others are launched one by one.
+  RoundBatch<kRoundBatchMax> batch;
+  batch.n_rounds = 0;
+  uint32_t version_before[kMaxDevices];  // the counters before the pending batch, should its launch fail
+  uint64_t step_count_before[kMaxDevices];
+  auto flush = [&]() -> int {
+    if (batch.n_rounds == 0) return HADFL_OK;
+    int rc;
+    {
+      DeviceGuard guard(h->device);
+      if (batch.n_rounds == 1) {
+        RoundBatch<1> one;
+        one.n_rounds = 1;
+        one.round[0] = batch.round[0];
+        rc = launch_round(h, one, lr);
+      } else {
+        rc = launch_round(h, batch, lr);
+      }
+    }
+    if (rc == HADFL_OK) {
+      h->stats_valid = true;
+      h->last_launch_rounds = batch.n_rounds;
+    } else {
+      memcpy(h->version, version_before, sizeof(version_before));
+      memcpy(h->step_count, step_count_before, sizeof(step_count_before));
+    }
+    batch.n_rounds = 0;
+    return rc;
+  };
   for (int32_t i = 0; i < n_rounds; ++i) {
     const int64_t r = first_round + i;
     const int32_t sync = sync_every > 0 && (r + 1) % sync_every == 0;
-    const int rc = hadfl_round(h, ids, steps + (int64_t)i * N, N, lr, r, nullptr, seed, k, sync, sel);
+    const int32_t *round_steps = steps + (int64_t)i * N;
+    RoundPlan pl;
+    int rc = plan_round(h, ids, round_steps, N, r, nullptr, seed, k, sync, pl);
+    if (rc != HADFL_OK) {
+      const int rc_flush = flush();  // what was planned before the bad round still runs
+      return rc_flush != HADFL_OK ? rc_flush : rc;
+    }
+    if (pl.crosses) {
+      rc = flush();
+      if (rc == HADFL_OK) rc = round_by_separate_calls(h, ids, round_steps, N, lr, nullptr, k, sync, pl.sel);
+    } else {
+      if (!batchable(h, pl)) rc = flush();
+      if (rc == HADFL_OK) {
+        if (batch.n_rounds == 0) {
+          memcpy(version_before, h->version, sizeof(version_before));
+          memcpy(step_count_before, h->step_count, sizeof(step_count_before));
+        }
+        batch.round[batch.n_rounds++] = pl.a;
+        commit_round(h, pl, k, sync);
+        if (!batchable(h, pl) || batch.n_rounds >= h->round_batch) rc = flush();
+      }
+    }
     if (rc != HADFL_OK) return rc;
     if (out_selected)
-      for (int j = 0; j < k; ++j) out_selected[(int64_t)i * k + j] = sel[j];
+      for (int j = 0; j < k; ++j) out_selected[(int64_t)i * k + j] = pl.sel[j];
   }
+  return flush();
+}
+
+int hadfl_set_round_batch(hadfl_handle *h, int32_t max_rounds) {
+  if (!h || max_rounds < 1 || max_rounds > kRoundBatchMax) return HADFL_ERR_INVALID;
+  h->round_batch = max_rounds;
+  return HADFL_OK;
+}
+
+int32_t hadfl_round_batch(const hadfl_handle *h) { return h ? h->round_batch : 0; }
+
+int hadfl_stats_read_round(hadfl_handle *h, int32_t back, float *out_norm2, float *out_div2) {
+  if (!h || !out_norm2 || !out_div2 || back < 0) return HADFL_ERR_INVALID;
+  if (back == 0) return hadfl_stats_read(h, out_norm2, out_div2);
+  if (!h->stats_valid || back >= h->last_launch_rounds) return HADFL_ERR_STATE;
+  DeviceGuard guard(h->device);
+  float buf[2 * kMaxDevices];
+  const int n = h->cfg.n_devices;
+  const float *src = h->d_round_stats + (size_t)(h->last_launch_rounds - 1 - back) * 2 * kMaxDevices;
+  HADFL_CUDA(h, cudaMemcpyAsync(buf, src, sizeof(float) * 2 * (size_t)n, cudaMemcpyDeviceToHost, h->stream));
+  HADFL_CUDA(h, cudaStreamSynchronize(h->stream));
+  HADFL_DEBUG_RESULT();
+  memcpy(out_norm2, buf, sizeof(float) * (size_t)n);
+  memcpy(out_div2, buf + n, sizeof(float) * (size_t)n);
   return HADFL_OK;
 }
 

@@ -944,9 +944,14 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 // (live = 0) take part in everything: their loads return zeros, their stores store nothing, and
 // what they compute is zeroed before it is summed.
 // Row sums: one shuffle per row and pack, then a shared-memory slot owned by the thread (fp32); at
-// the end of the block, per row, a fixed-order sum over the warps and a butterfly over each
-// half-warp (fp64) -> partials[value][block]; two-level last-ticket finish.  Deterministic.
+// the end of a chunk's round, per row, a fixed-order sum over the warps and a butterfly over each
+// half-warp (fp64), added to the block's sums of that round; at the end of the block
+// partials[round][value][block] and a two-level last-ticket finish per round.  Deterministic.
 // Dynamic shared memory: n * kThreads floats.  64 registers: four resident blocks per SM.
+// NR > 1: the launch takes a batch of up to NR consecutive rounds.  A block carries its chunk
+// through all of them before it moves on (chunk loop outside, round loop inside), so from the
+// second round on the rows come from L2 and not from HBM, and every round still leaves its own
+// statistics.  Results are those of the rounds launched one by one, bit for bit.
 // PF = true is a second build that issues the next row's loads before the current row's steps
 // (80 registers, three resident blocks).  With bf16 parameters a row is 48 bytes per thread or
 // less, and when every device runs one or two steps the launch is bound by how many bytes are in
@@ -977,17 +982,39 @@ __device__ __forceinline__ void add_row_sums(float *s_acc, int j, float n2, floa
 
 constexpr int kRoundBlocksPerSM = 4;
 
-template <typename WT, typename MT, typename Gen, int E, int RM, bool PF>
+// A batch of consecutive rounds for one launch.  Every operation of a round is elementwise in the
+// parameter index and the selections are known to the host beforehand, so a thread can take its
+// pack through several rounds back to back: what it wrote in one round it reads back in the next
+// (the same thread, the same addresses, program order), while the lines are still in L2.
+template <int NR>
+struct RoundBatch {
+  int32_t n_rounds;  // 1 <= n_rounds <= NR
+  RoundArgs round[NR];
+};
+constexpr int kRoundBatchMax = 8;
+
+// Scratch of the fused round kernel, per round of a batch.
+struct RoundScratch {
+  double *partials;            // [round][2 n][blocks]
+  double *group_partials;      // [round][2 n][groups]
+  unsigned int *tickets;       // [round][1 + groups]: the round's ticket, then one per group
+  float *out_rounds;           // [round][2 kMaxDevices]: the statistics of every round of the batch
+  float *out;                  // [2 kMaxDevices]: the statistics of the batch's last round
+};
+
+template <typename WT, typename MT, typename Gen, int E, int RM, bool PF, int NR>
 __global__ void __launch_bounds__(kThreads, PF ? kRoundBlocksPerSM - 1 : kRoundBlocksPerSM)
-k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, PhiloxKeys keys,
-        StepConsts k, double *__restrict__ partials, double *__restrict__ group_partials,
-        unsigned int *__restrict__ group_tickets, unsigned int *__restrict__ ticket,
-        float *__restrict__ out) {
+k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundBatch<NR> b, PhiloxKeys keys,
+        StepConsts k, RoundScratch scratch) {
   constexpr int kWarps = kThreads / 32;
-  extern __shared__ float s_acc[];  // [a.n][kThreads]: per-thread row sums
+  extern __shared__ float s_acc[];  // [n][kThreads]: per-thread row sums of the round in hand
+  __shared__ double s_part[NR][2 * kMaxDevices];  // the block's sums, per round
   __shared__ bool s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int j = 0; j < a.n; ++j) s_acc[j * kThreads + threadIdx.x] = 0.f;
+  const int n_dev = b.round[0].n;
+  for (int j = 0; j < n_dev; ++j) s_acc[j * kThreads + threadIdx.x] = 0.f;
+  for (int t = threadIdx.x; t < NR * 2 * kMaxDevices; t += kThreads) (&s_part[0][0])[t] = 0.0;
+  __syncthreads();
 
   const int64_t n_packs = (n_params + E - 1) / E;
   const int64_t n_chunks = (n_packs + kThreads - 1) / kThreads;
@@ -1002,97 +1029,125 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
       char *wp = reinterpret_cast<char *>(w) + p * (int64_t)(E * sizeof(WT));
       char *mp = reinterpret_cast<char *>(m) + p * (int64_t)(E * sizeof(MT));
 
-      // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
-      // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
-      // 0).  fp32 values are updated in the registers they were loaded into.
-      // PF: the next row's loads are issued before this row's steps (see the kernel's header).
-      RawPack<WT, E> rw_next;
-      RawPack<MT, E> rm_next;
-      auto fetch = [&](int j) {
-        ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw_next);
-        if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm_next);
-      };
-      if constexpr (PF) fetch(0);
-      auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
-        RawPack<WT, E> rw;
-        RawPack<MT, E> rm;
-        if constexpr (PF) {
-          rw = rw_next;
-          rm = rm_next;
-          if (j + 1 < a.n) fetch(j + 1);
-        } else {
-          ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
-        }
-        const bool stepped = a.r[j].steps > 0;
-        if (stepped) {
-          if constexpr (!PF) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
-          float mv[E];
-          unpack(rw, wv);
-          unpack(rm, mv);
-          sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
-          if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
-          st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
-#pragma unroll
-          for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
-          if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
-#pragma unroll
-            for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
+      auto do_round = [&](const RoundArgs &a, const int r) {
+        // Row j as it is after its local steps: loads w (and m when the row runs steps), runs the
+        // steps, stores the momentum, and leaves in wv what the row now holds (as stored; dead lanes
+        // 0).  fp32 values are updated in the registers they were loaded into.
+        // PF: the next row's loads are issued before this row's steps (see the kernel's header).
+        RawPack<WT, E> rw_next;
+        RawPack<MT, E> rm_next;
+        auto fetch = [&](int j) {
+          ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw_next);
+          if (a.r[j].steps > 0) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm_next);
+        };
+        if constexpr (PF) fetch(0);
+        auto row_after_steps = [&](int j, float (&wv)[E]) -> bool {
+          RawPack<WT, E> rw;
+          RawPack<MT, E> rm;
+          if constexpr (PF) {
+            rw = rw_next;
+            rm = rm_next;
+            if (j + 1 < a.n) fetch(j + 1);
+          } else {
+            ld_raw(at_row<WT>(wp, a.r[j].w_off), live, rw);
           }
-        } else {
-          unpack(rw, wv);
-        }
-        return stepped;
-      };
+          const bool stepped = a.r[j].steps > 0;
+          if (stepped) {
+            if constexpr (!PF) ld_raw(at_row<MT>(mp, a.r[j].m_off), live, rm);
+            float mv[E];
+            unpack(rw, wv);
+            unpack(rm, mv);
+            sgd_steps<Gen, E / 4>(wv, mv, gp, a.r[j], keys, k);
+            if constexpr (RM == 1) round_stochastic<MT, E / 4>(wv, mv, p, a.r[j], keys);
+            st_pack_any(at_row<MT>(mp, a.r[j].m_off), 0, live, mv);
+#pragma unroll
+            for (int i = 0; i < E; ++i) wv[i] = as_stored(wv[i], w);
+            if (live < E) {  // the ragged last pack of a row and the lanes beyond it: dead lanes stay 0
+#pragma unroll
+              for (int i = 0; i < E; ++i) wv[i] = i < live ? wv[i] : 0.f;
+            }
+          } else {
+            unpack(rw, wv);
+          }
+          return stepped;
+        };
 
-      // ---- the selected devices in draw order: acc = a_0 w_0, then acc = fma(a_j, w_j, acc)
-      float acc[E];
-      {
-        float wv[E];
-        row_after_steps(0, wv);
-        const float a0 = a.a[0];
+        // ---- the selected devices in draw order: acc = a_0 w_0, then acc = fma(a_j, w_j, acc)
+        float acc[E];
+        {
+          float wv[E];
+          row_after_steps(0, wv);
+          const float a0 = a.a[0];
 #pragma unroll
-        for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
-      }
-      for (int j = 1; j < a.k; ++j) {
-        float wv[E];
-        row_after_steps(j, wv);
-        const float aj = a.a[j];
-#pragma unroll
-        for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
-      }
-      {
-        float n2 = 0.f;
-#pragma unroll
-        for (int i = 0; i < E; ++i) {
-          acc[i] = as_stored(acc[i], w);
-          n2 = fmaf(acc[i], acc[i], n2);
+          for (int i = 0; i < E; ++i) acc[i] = __fmul_rn(a0, wv[i]);
         }
-        // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
-        if (a.k > 1 || a.r[0].steps > 0)
-          for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
-        add_row_sums(s_acc, a.k - 1, n2, 0.f, lane);  // one value for all selected devices
-      }
-      // ---- the other devices: keep their own model, or receive the aggregate
-      for (int j = a.k; j < a.n; ++j) {
-        float wv[E];
-        const bool stepped = row_after_steps(j, wv);
-        if (a.write_all == 1) {
+        for (int j = 1; j < a.k; ++j) {
+          float wv[E];
+          row_after_steps(j, wv);
+          const float aj = a.a[j];
 #pragma unroll
-          for (int i = 0; i < E; ++i) wv[i] = acc[i];
-        } else if (a.write_all == 2) {
-#pragma unroll
-          for (int i = 0; i < E; ++i)
-            wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
+          for (int i = 0; i < E; ++i) acc[i] = fmaf(aj, wv[i], acc[i]);
         }
-        if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
-        float n2 = 0.f, d2 = 0.f;
+        {
+          float n2 = 0.f;
 #pragma unroll
-        for (int i = 0; i < E; ++i) {
-          const float d = wv[i] - acc[i];
-          n2 = fmaf(wv[i], wv[i], n2);
-          d2 = fmaf(d, d, d2);
+          for (int i = 0; i < E; ++i) {
+            acc[i] = as_stored(acc[i], w);
+            n2 = fmaf(acc[i], acc[i], n2);
+          }
+          // a single selected device that ran no steps already holds the aggregate (a_0 = 1)
+          if (a.k > 1 || a.r[0].steps > 0)
+            for (int t = 0; t < a.k; ++t) st_pack_any(at_row<WT>(wp, a.r[t].w_off), 0, live, acc);
+          add_row_sums(s_acc, a.k - 1, n2, 0.f, lane);  // one value for all selected devices
         }
-        add_row_sums(s_acc, j, n2, d2, lane);
+        // ---- the other devices: keep their own model, or receive the aggregate
+        for (int j = a.k; j < a.n; ++j) {
+          float wv[E];
+          const bool stepped = row_after_steps(j, wv);
+          if (a.write_all == 1) {
+#pragma unroll
+            for (int i = 0; i < E; ++i) wv[i] = acc[i];
+          } else if (a.write_all == 2) {
+#pragma unroll
+            for (int i = 0; i < E; ++i)
+              wv[i] = as_stored(fmaf(a.beta, acc[i], __fmul_rn(a.one_minus_beta, wv[i])), w);
+          }
+          if (stepped || a.write_all) st_pack_any(at_row<WT>(wp, a.r[j].w_off), 0, live, wv);
+          float n2 = 0.f, d2 = 0.f;
+#pragma unroll
+          for (int i = 0; i < E; ++i) {
+            const float d = wv[i] - acc[i];
+            n2 = fmaf(wv[i], wv[i], n2);
+            d2 = fmaf(d, d, d2);
+          }
+          add_row_sums(s_acc, j, n2, d2, lane);
+        }
+        // ---- block: fold the per-thread slots of every visit index j >= k - 1 into the block's
+        // sums of this round and clear them.  Warp w takes the visit indices k - 1 + w,
+        // k - 1 + w + 8, ...: each lane adds the slots of the threads that share its lane index
+        // (one per warp, in warp order; lower half-warps hold norms, upper halves distances), then a
+        // butterfly over the half-warp finishes the two sums.
+        __syncthreads();
+        for (int j = a.k - 1 + warp; j < a.n; j += kWarps) {
+          float v = 0.f;
+#pragma unroll
+          for (int wi = 0; wi < kWarps; ++wi) {
+            v += s_acc[j * kThreads + wi * 32 + lane];
+            s_acc[j * kThreads + wi * 32 + lane] = 0.f;
+          }
+          double d = (double)v;
+#pragma unroll
+          for (int off = 8; off > 0; off >>= 1) d += __shfl_xor_sync(0xFFFFFFFFu, d, off);
+          if ((lane & 15) == 0) s_part[r][2 * j + (lane >> 4)] += d;  // value = 2 * visit index + which
+        }
+        __syncthreads();
+      };
+      // A launch of a single round reads its arguments at constant addresses (the compiler then
+      // keeps the row descriptors on the uniform datapath); a batch indexes them by the round.
+      if constexpr (NR == 1) {
+        do_round(b.round[0], 0);
+      } else {
+        for (int r = 0; r < b.n_rounds; ++r) do_round(b.round[r], r);
       }
     };
     if ((chunk + 1) * kThreads * E <= n_params)
@@ -1100,36 +1155,36 @@ k_round(WT *__restrict__ w, MT *__restrict__ m, int64_t n_params, RoundArgs a, P
     else
       do_chunk(std::false_type{});
   }
-  // ---- block: sum the per-thread slots of every visit index j >= k - 1.  Warp w takes the visit
-  // indices k - 1 + w, k - 1 + w + 8, ...: each lane adds the slots of the threads that share its
-  // lane index (one per warp, in warp order; lower half-warps hold norms, upper halves distances),
-  // then a butterfly over the half-warp finishes the two sums.
-  __syncthreads();
-  for (int j = a.k - 1 + warp; j < a.n; j += kWarps) {
-    float v = 0.f;
-#pragma unroll
-    for (int wi = 0; wi < kWarps; ++wi) v += s_acc[j * kThreads + wi * 32 + lane];
-    double d = (double)v;
-#pragma unroll
-    for (int off = 8; off > 0; off >>= 1) d += __shfl_xor_sync(0xFFFFFFFFu, d, off);
-    // partials[value][block]; value = 2 * visit index + which
-    double *slot = partials + (int64_t)(2 * j + (lane >> 4)) * gridDim.x + blockIdx.x;
-    if ((lane & 15) == 0 && access_ok(slot, 8)) *slot = d;
-  }
-  const int n_dev = a.n, ksel = a.k;
-  finish_two_level(partials + (int64_t)2 * (ksel - 1) * gridDim.x, group_partials, 2 * (n_dev - ksel + 1),
-                   group_tickets, ticket, &s_last, [&](int t, double sum) {
-    const int j = ksel - 1 + (t >> 1), which = t & 1;
-    if (j == ksel - 1) {  // the selected devices share one norm and are at distance 0
-      for (int q = 0; q < ksel; ++q) {
-        float *o = out + which * n_dev + a.r[q].row;
-        if (access_ok(o, 4)) *o = which ? 0.f : (float)sum;
-      }
-    } else {
-      float *o = out + which * n_dev + a.r[j].row;
-      if (access_ok(o, 4)) *o = (float)sum;
+  // ---- launch: per round, partials[value][block] and the two-level last-ticket finish
+  const int n_blocks = (int)gridDim.x;
+  const int n_groups = (n_blocks + kFinishGroup - 1) / kFinishGroup;
+  for (int r = 0; r < (NR == 1 ? 1 : b.n_rounds); ++r) {
+    const RoundArgs &a = b.round[NR == 1 ? 0 : r];
+    const int ksel = a.k;
+    double *partials = scratch.partials + (int64_t)r * 2 * n_dev * n_blocks;
+    double *group_partials = scratch.group_partials + (int64_t)r * 2 * n_dev * n_groups;
+    unsigned int *tickets = scratch.tickets + (int64_t)r * (1 + n_groups);
+    float *out_r = scratch.out_rounds + r * 2 * kMaxDevices;
+    const bool is_last_round = r + 1 == (NR == 1 ? 1 : b.n_rounds);
+    auto put = [&](int at, float v) {  // every round's statistics; the last round's also where hadfl_stats puts them
+      if (access_ok(out_r + at, 4)) out_r[at] = v;
+      if (is_last_round && access_ok(scratch.out + at, 4)) scratch.out[at] = v;
+    };
+    for (int t = 2 * (ksel - 1) + threadIdx.x; t < 2 * n_dev; t += kThreads) {
+      double *slot = partials + (int64_t)t * n_blocks + blockIdx.x;
+      if (access_ok(slot, 8)) *slot = s_part[r][t];
     }
-  });
+    finish_two_level(partials + (int64_t)2 * (ksel - 1) * n_blocks,
+                     group_partials + (int64_t)2 * (ksel - 1) * n_groups, 2 * (n_dev - ksel + 1),
+                     tickets + 1, tickets, &s_last, [&](int t, double sum) {
+      const int j = ksel - 1 + (t >> 1), which = t & 1;
+      if (j == ksel - 1) {  // the selected devices share one norm and are at distance 0
+        for (int q = 0; q < ksel; ++q) put(which * n_dev + a.r[q].row, which ? 0.f : (float)sum);
+      } else {
+        put(which * n_dev + a.r[j].row, (float)sum);
+      }
+    });
+  }
 }
 
 // ------------------------------------------------------------------------------------------

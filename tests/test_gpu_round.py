@@ -207,3 +207,102 @@ def test_fused_round_counter_crossing_falls_back_to_separate_kernels():
     assert_same_state(fused, plain, 3)
     fused.close()
     plain.close()
+
+
+# ---- several rounds per launch ---------------------------------------------------------------------
+def _launches(ar, fn):
+    before = ar.h.launch_count()
+    out = fn()
+    return out, ar.h.launch_count() - before
+
+
+@pytest.mark.parametrize("dtype,m_dtype,rounding", [(0, 0, 0), (1, 0, 0), (1, 1, 0), (1, 0, 1), (1, 1, 1)])
+@pytest.mark.parametrize("n,P,k,sync_every,beta", [(4, 100_003, 2, 0, 1.0), (8, 70_001, 4, 3, 0.5),
+                                                  (16, 9_999, 1, 4, 1.0), (32, 2_049, 16, 0, 1.0), (5, 7, 5, 2, 0.25)])
+def test_batched_rounds_equal_the_rounds_launched_one_by_one(n, P, k, sync_every, beta, dtype, m_dtype, rounding):
+    """A small arena: hadfl_rounds puts up to 8 rounds into one launch.  Parameters, momentum, counters,
+    selections and EVERY round's statistics must equal those of single launches, bit for bit."""
+    steps = tuple((5 * i + 1) % 4 for i in range(n))  # 0 .. 3 steps, some devices idle
+    wl = wl_of(n, P, k, dtype=dtype, steps=steps, sync_every=sync_every, sync_beta=beta, m_dtype=m_dtype,
+               rounding=rounding)
+    single, batched = runtime.Arena(wl), runtime.Arena(wl)
+    assert batched.h.round_batch() == 8
+    single.h.set_round_batch(1)
+    stats_single = []
+    want = []
+    for r in range(19):
+        want.append(single.run_round_fused(r))
+        stats_single.append(single.h.stats_read())
+    got = []
+    for first, count in ((0, 8), (8, 8), (16, 3)):
+        sel, launches = _launches(batched, lambda: batched.run_rounds_fused(first, count))
+        assert launches == 1
+        got.append(sel)
+        for back in range(count):
+            a = batched.h.stats_read_round(back)
+            b = stats_single[first + count - 1 - back]
+            assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]), (first, back)
+        with pytest.raises(binding.HadflError):
+            batched.h.stats_read_round(count)
+    assert np.array_equal(np.concatenate(got), np.stack(want))
+    assert_same_state(single, batched, n)
+    # the same through hadfl_rounds with batching switched off: one launch per round
+    off = runtime.Arena(wl)
+    off.h.set_round_batch(1)
+    sel, launches = _launches(off, lambda: off.run_rounds_fused(0, 19))
+    assert launches == 19 and np.array_equal(sel, np.stack(want))
+    assert_same_state(single, off, n)
+    for ar in (single, batched, off):
+        ar.h.debug_check()  # debug build: no kernel skipped an out-of-range access (no-op otherwise)
+        ar.close()
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_batching_rule_on_an_arena_larger_than_the_small_arena_bound(dtype):
+    """Beyond 64 MiB only rounds in which no device runs more than two steps are batched."""
+    n, P, k = 8, 1_300_003, 4  # fp32: 83 MB, bf16 parameters: 62 MB of parameters and momentum
+    if dtype == 1:
+        P = 2_000_003  # 96 MB
+    light = np.array([1, 2, 0, 1, 2, 2, 1, 1], dtype=np.int32)
+    heavy = np.array([1, 3, 0, 1, 2, 2, 1, 1], dtype=np.int32)
+    steps = np.stack([light, light, light, heavy, light, light, heavy, heavy, light])
+    # launches: [0 1 2] [3] [4 5] [6] [7] [8]
+    wl = Workload("rule", n, P, k, 9, "fixed", tuple(light), grad_std=1e-2, dtype=dtype, seed=workloads.BASE_SEED + 77,
+                  sync_every=4)
+    single, batched = runtime.Arena(wl), runtime.Arena(wl)
+    want = np.stack([single.h.round(single.ids, steps[r], wl.lr, r, k, single.select_seed,
+                                    sync_all=(r + 1) % 4 == 0) for r in range(9)])
+    got, launches = _launches(batched, lambda: batched.h.rounds(0, steps, wl.lr, k, batched.select_seed, 4))
+    assert launches == 6
+    assert np.array_equal(got, want)
+    batched.h.synchronize()
+    single.h.synchronize()
+    assert torch.equal(single.w, batched.w) and torch.equal(single.m, batched.m)
+    a, b = single.h.stats_read(), batched.h.stats_read()
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    batched.h.set_round_batch(2)
+    _, launches = _launches(batched, lambda: batched.h.rounds(9, steps[:3], wl.lr, k, batched.select_seed, 4))
+    assert launches == 2
+    for bad in (0, 9, -1):
+        with pytest.raises(binding.HadflError):
+            batched.h.set_round_batch(bad)
+    assert batched.h.round_batch() == 2
+    single.close()
+    batched.close()
+
+
+def test_batched_rounds_with_a_step_counter_crossing_2_to_the_32():
+    """The round in which a counter crosses a multiple of 2^32 leaves the batch (separate kernels); the
+    rounds before and after it are batched around it."""
+    wl = wl_of(3, 4_099, 2, steps=(2, 1, 3))
+    batched, plain = runtime.Arena(wl), runtime.Arena(wl)
+    start = np.array([2**32 - 5, 5, 2**33 - 7], dtype=np.uint64)  # device 0 crosses in round 2, device 2 in round 2
+    for ar in (batched, plain):
+        ar.h.set_versions(step_counts=start)
+    got, launches = _launches(batched, lambda: batched.run_rounds_fused(0, 6))
+    want = np.stack([plain.run_round(r) for r in range(6)])
+    assert np.array_equal(got, want)
+    assert_same_state(batched, plain, 3)
+    assert launches > 2  # two batches and the kernels of the crossing round in between
+    batched.close()
+    plain.close()
