@@ -321,13 +321,22 @@ def measure_case(wl, rounds, peak, frac_key, warmup=3):
     r += rounds
     # rounds/s with 8 rounds enqueued per library call (hadfl_rounds): small vectors then show the
     # kernel and not the per-call overhead of the caller, while the launch queue stays shallow
-    torch.cuda.synchronize()
-    start.record()
-    for i in range(0, 2 * rounds, 8):
-        arena.run_rounds_fused(r + i, min(8, 2 * rounds - i))
-    end.record()
-    torch.cuda.synchronize()
-    fused_wall_ms = start.elapsed_time(end) / (2 * rounds)
+    def rounds_by_calls_of_8(r0):
+        launches0 = h.launch_count()
+        torch.cuda.synchronize()
+        start.record()
+        for i in range(0, 2 * rounds, 8):
+            arena.run_rounds_fused(r0 + i, min(8, 2 * rounds - i))
+        end.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(end) / (2 * rounds), 2 * rounds / (h.launch_count() - launches0)
+    fused_wall_ms, rounds_per_launch = rounds_by_calls_of_8(r)
+    r += 2 * rounds
+    # where the library put several rounds into one launch: the same with one launch per round
+    single_wall_ms = fused_wall_ms
+    if rounds_per_launch > 1:
+        h.set_round_batch(1)
+        single_wall_ms, _ = rounds_by_calls_of_8(r)
     grid = h.round_grid()
     arena.close()
     nbytes = {"local_step": N * P * 2 * (ew + em), "aggregate": 2 * k * P * ew, "stats": N * P * ew,
@@ -337,6 +346,7 @@ def measure_case(wl, rounds, peak, frac_key, warmup=3):
            "storage": ("bf16" if wl.dtype else "fp32") + ("+bf16 m" if wl.m_dtype else ""),
            "mean_steps_per_device": mean_steps, "arena_mb": N * P * (ew + em) / 1e6,
            "rounds_per_s": 1e3 / fused_wall_ms, "round_ms": fused_wall_ms, "round_grid_blocks": grid,
+           "rounds_per_launch": rounds_per_launch, "rounds_per_s_one_round_per_launch": 1e3 / single_wall_ms,
            "separate_calls_rounds_per_s": 1e3 / (ms["local_step"] + ms["aggregate"] + ms["stats"]),
            "hbm_bound": bool(N * P * (ew + em) > 126e6),
            "kernels": {"round": gbs_entry(nbytes["round"], fused_ms, peak, frac_key)}}
@@ -424,14 +434,16 @@ def print_tables(path):
         return "%.1f | %.0f (%.0f / %.0f)" % (k["avg_ms"] * 1e3, k["achieved_gbs"], 100 * k[key], 100 * k["frac_of_8TBs"])
     print("GB/s = algorithmic bytes / time; percentages: of the %s %.0f GB/s / of the nominal 8000 GB/s.\n" % (sw["peak_kind"], peak))
     print("| workload | N | P | k | storage | mean steps | K1 µs | K1 GB/s (% meas / % 8T) | K2 µs | K2 GB/s (%/%) | K3 µs | K3 GB/s (%/%) "
-          "| separate calls rounds/s | fused `hadfl_round` µs | fused GB/s (%/%) | fused rounds/s | G element-steps/s |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+          "| separate calls rounds/s | fused `hadfl_round` µs | fused GB/s (%/%) | fused rounds/s, one round per launch "
+          "| `hadfl_rounds` rounds/s (rounds per launch) | G element-steps/s |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for p in sw["points"]:
         ks = p["kernels"]
-        print("| %s | %d | %d | %d | %s | %.2f | %s | %s | %s | %.0f | %s | %.0f | %.0f |" % (
+        print("| %s | %d | %d | %d | %s | %.2f | %s | %s | %s | %.0f | %s | %.0f | %.0f (%.3g) | %.0f |" % (
             p["workload"], p["N"], p["P"], p["k"], p["storage"], p["mean_steps_per_device"], cell(ks["local_step"]),
             cell(ks["aggregate"]), cell(ks["stats"]), p["separate_calls_rounds_per_s"], cell(ks["round"]),
-            p["rounds_per_s"], ks["round"]["gelem_steps_per_s"]))
+            p["rounds_per_s_one_round_per_launch"], p["rounds_per_s"], p["rounds_per_launch"],
+            ks["round"]["gelem_steps_per_s"]))
     if sw.get("sync"):
         print("\n| workload | N | P | receivers | storage | broadcast µs | GB/s (%/%) | integrate µs | GB/s (%/%) |")
         print("|---|---|---|---|---|---|---|---|---|")
@@ -710,7 +722,8 @@ def run_profile_case(a):
     stay at a few hundred MB so that a multi-pass capture ends quickly.  Launch order per repetition:
     local update once per entry of --pc-steps (all devices that many steps), aggregation of k
     devices, statistics, broadcast to the other devices, the same as a mix (beta = 1/2).  With
-    --pc-fused: one hadfl_round launch per entry of --pc-steps instead."""
+    --pc-fused: one hadfl_round launch per entry of --pc-steps instead; with --pc-batch R also one
+    hadfl_rounds call of R rounds per entry (one launch of R rounds where the library batches them)."""
     from paper_2111_08274_b200 import runtime
     wl = workloads.Workload("profile", a.pc_n, a.pc_p, a.pc_k, 1, "fixed", (1,) * a.pc_n, dtype=a.pc_dtype,
                             seed=workloads.BASE_SEED)
@@ -723,6 +736,8 @@ def run_profile_case(a):
         if a.pc_fused:
             for s in steps:
                 ar.h.round(ids, np.full(a.pc_n, s, dtype=np.int32), wl.lr, rep, a.pc_k, 1)
+            for s in steps if a.pc_batch > 1 else ():
+                ar.h.rounds(100 * rep, np.full((a.pc_batch, a.pc_n), s, dtype=np.int32), wl.lr, a.pc_k, 1)
             continue
         for s in steps:
             ar.h.local_step(ids, np.full(a.pc_n, s, dtype=np.int32), wl.lr)
@@ -758,6 +773,7 @@ def main():
     ap.add_argument("--pc-dtype", type=int, default=0)
     ap.add_argument("--pc-reps", type=int, default=2)
     ap.add_argument("--pc-fused", action="store_true", help="hadfl_round instead of the separate calls")
+    ap.add_argument("--pc-batch", type=int, default=0, help="with --pc-fused: also hadfl_rounds calls of that many rounds")
     args = ap.parse_args()
     if args.no_sweep:
         args.sweep = "none"

@@ -217,7 +217,8 @@ int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const i
  * second round on the replicas are read from L2 instead of HBM.  Results - parameters, momentum,
  * counters, selections, every round's statistics - are those of the rounds launched one by one,
  * bit for bit.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
- * steps, or the whole arena is at most 64 MiB) and launches the others singly.
+ * steps and rounding is to nearest even, or the whole arena - parameters and momentum of all
+ * devices - is at most 64 MiB) and launches the others singly.
  * hadfl_set_round_batch: the most rounds per launch, 1 .. 8 (default 8; 1 = never batch);
  * HADFL_ERR_INVALID outside that range.  hadfl_round_batch returns the setting (0 for NULL). */
 int hadfl_set_round_batch(hadfl_handle *h, int32_t max_rounds);

@@ -762,13 +762,15 @@ int round_by_separate_calls(hadfl_handle *h, const int32_t *device_ids, const in
 // batch pays where a round is bound by memory or by the launch itself: every device runs at most
 // kRowPerBlockMaxSteps steps, or the arena is small against the L2.  With more steps per device
 // the rounds are bound by arithmetic and the batch's indexed arguments cost what L2 saves
-// (measured: 0 ... -3 %), so those rounds are launched one by one.
+// (measured: 0 ... -3 %), so those rounds are launched one by one; the same holds for stochastic
+// rounding, which draws a second random block per pack and call (measured: -3 ... -5 %).
 constexpr size_t kBatchSmallArenaBytes = (size_t)64 << 20;
 
 bool batchable(const hadfl_handle *h, const RoundPlan &pl) {
   if (h->round_batch <= 1) return false;
   const size_t arena = (size_t)h->cfg.n_devices * (size_t)h->cfg.n_params * (elem_size(h) + m_elem_size(h));
   if (arena <= kBatchSmallArenaBytes) return true;
+  if (h->cfg.rounding == HADFL_ROUND_STOCHASTIC) return false;
   for (int i = 0; i < h->cfg.n_devices; ++i)
     if (pl.row_steps[i] > kRowPerBlockMaxSteps) return false;
   return true;

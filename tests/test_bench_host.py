@@ -57,6 +57,7 @@ def test_table_printer_reads_a_saved_line(bench, tmp_path, capsys):
     k["gelem_steps_per_s"] = 400.0
     point = {"workload": "c5_p24_fp32", "N": 16, "P": 1 << 24, "k": 4, "storage": "fp32",
              "mean_steps_per_device": 1.0, "rounds_per_s": 1500.0, "separate_calls_rounds_per_s": 1100.0,
+             "rounds_per_launch": 8.0, "rounds_per_s_one_round_per_launch": 1400.0,
              "kernels": {"round": k, "local_step": k, "aggregate": k, "stats": k}}
     line = {"sweep": {"peak_gbs": 6464.3, "peak_kind": "measured", "points": [point]}}
     path = tmp_path / "line.json"
@@ -64,3 +65,4 @@ def test_table_printer_reads_a_saved_line(bench, tmp_path, capsys):
     bench.print_tables(str(path))
     out = capsys.readouterr().out
     assert "| c5_p24_fp32 | 16 | 16777216 | 4 | fp32 | 1.00 |" in out and "5000 (77 / 62)" in out
+    assert "| 1400 | 1500 (8) |" in out

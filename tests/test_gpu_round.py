@@ -289,6 +289,12 @@ def test_batching_rule_on_an_arena_larger_than_the_small_arena_bound(dtype):
     assert batched.h.round_batch() == 2
     single.close()
     batched.close()
+    if dtype == 1:  # stochastic rounding draws a second random block per pack: launched one by one
+        from dataclasses import replace
+        sr = runtime.Arena(replace(wl, rounding=1))
+        _, launches = _launches(sr, lambda: sr.h.rounds(0, steps[:3], wl.lr, k, sr.select_seed, 4))
+        assert launches == 3
+        sr.close()
 
 
 def test_batched_rounds_with_a_step_counter_crossing_2_to_the_32():
