@@ -73,3 +73,48 @@ def test_full_size_mixed_synchronisation_whole_arena_bit_for_bit():
     from dataclasses import replace
     wl = replace(workloads.c3(), sync_every=2, sync_beta=0.25)
     run_both(wl, 4)
+
+
+@pytest.mark.parametrize("name,rounds", [("c5_p27_fp32", 9), ("c5_p26_bf16", 9), ("c5_p24_fp32", 10), ("c5_p22_bf16", 17)])
+def test_full_size_batched_rounds_whole_arena_bit_for_bit(name, rounds):
+    """One step per device: hadfl_rounds puts 8 rounds into each launch.  Against one launch per round, over
+    the whole arena; from 2^26 parameters up the blocks stride over several chunks, each taken through the
+    whole batch before the next."""
+    from dataclasses import replace
+    wl = replace(workloads.by_name(name), sync_every=4)
+    batched, single = runtime.Arena(wl), runtime.Arena(wl)
+    single.h.set_round_batch(1)
+    before = batched.h.launch_count()
+    sb = batched.run_rounds_fused(0, rounds)
+    assert batched.h.launch_count() - before == (rounds + 7) // 8
+    ss = single.run_rounds_fused(0, rounds)
+    assert np.array_equal(sb, ss)
+    batched.h.synchronize()
+    single.h.synchronize()
+    assert torch.equal(batched.w, single.w), "parameters differ between batched and single launches"
+    assert torch.equal(batched.m, single.m), "momentum differs between batched and single launches"
+    vb, vs = batched.h.get_versions(), single.h.get_versions()
+    assert np.array_equal(vb[0], vs[0]) and np.array_equal(vb[1], vs[1])
+    a, b = batched.h.stats_read(), single.h.stats_read()
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    batched.h.debug_check()
+    batched.close()
+    single.close()
+
+
+def test_full_size_batched_rounds_against_the_oracle(oracle):
+    """The ResNet-18 size with one step per device, 8 devices: 11 rounds in two launches (8 + 3), sampled
+    columns against the oracle."""
+    from dataclasses import replace
+    wl = replace(workloads.c2(), name="c2_steps1", steps_rule="fixed", steps_fixed=(1,) * 8, sync_every=5)
+    groups = workloads.sample_groups(wl.n_params, 4_000, 1_024, seed=91)
+    arena = runtime.Arena(wl)
+    sim = make_sim(oracle, wl, groups)
+    before = arena.h.launch_count()
+    sel = arena.run_rounds_fused(0, 11)
+    assert arena.h.launch_count() - before == 2
+    for r in range(11):
+        assert np.array_equal(sel[r], oracle_round(sim, wl, r)), r
+    assert np.array_equal(arena.h.get_versions()[0], sim.get_versions()[0])
+    compare_sample(arena, sim, groups, "c2_steps1 batched")
+    arena.close()
