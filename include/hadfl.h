@@ -215,14 +215,19 @@ int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const i
  * beforehand, so hadfl_rounds may hand several consecutive rounds to ONE launch of the fused kernel:
  * a block takes its columns through all of them before it moves to the next columns, and from the
  * second round on the replicas are read from L2 instead of HBM.  Results - parameters, momentum,
- * counters, selections, every round's statistics - are those of the rounds launched one by one,
- * bit for bit.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
+ * counters, selections - are those of the rounds launched one by one, bit for bit; so are every
+ * round's statistics, except that large fp32 arenas whose devices all run one step are taken in
+ * packs of half the width, which sums the statistics in a different (equally fixed) order: they
+ * then agree to rounding.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
  * steps and rounding is to nearest even, or the whole arena - parameters and momentum of all
  * devices - is at most 64 MiB) and launches the others singly.
  * hadfl_set_round_batch: the most rounds per launch, 1 .. 8 (default 8; 1 = never batch);
  * HADFL_ERR_INVALID outside that range.  hadfl_round_batch returns the setting (0 for NULL). */
 int hadfl_set_round_batch(hadfl_handle *h, int32_t max_rounds);
 int32_t hadfl_round_batch(const hadfl_handle *h);
+/* Columns per thread (8, or 4 for the half-width packs above) in the most recent launch of the fused
+ * round kernel; 0 before the first one or for NULL.  For tests and logs. */
+int32_t hadfl_last_round_pack(const hadfl_handle *h);
 
 /* The statistics that the fused kernel left for the round `back` rounds before the last one of its
  * most recent launch (back = 0: the last round, the same as hadfl_stats_read).  A launch keeps the

@@ -97,6 +97,7 @@ SIGNATURES = {
     "hadfl_round_grid": (C.c_int32, [_H]),
     "hadfl_set_round_batch": (C.c_int, [_H, C.c_int32]),
     "hadfl_round_batch": (C.c_int32, [_H]),
+    "hadfl_last_round_pack": (C.c_int32, [_H]),
     "hadfl_stats_read_round": (C.c_int, [_H, C.c_int32, _f32p, _f32p]),
     "hadfl_selection_probs": (C.c_int, [_f64p, _u8p, C.c_int32, _f64p]),
     "hadfl_selection_draw": (C.c_int, [_f64p, _u8p, C.c_int32, C.c_int64, C.c_uint64, C.c_int32, _i32p]),
@@ -412,6 +413,9 @@ class Hadfl:
 
     def round_batch(self):
         return int(self._lib.hadfl_round_batch(self._h))
+
+    def last_round_pack(self):
+        return int(self._lib.hadfl_last_round_pack(self._h))
 
     def debug_philox(self, counters, key):
         c = _arr(counters, np.uint32).reshape(-1, 4)

@@ -952,6 +952,10 @@ k_stats(const WT *__restrict__ w, int64_t stride, int64_t n_params, int n_device
 // through all of them before it moves on (chunk loop outside, round loop inside), so from the
 // second round on the rows come from L2 and not from HBM, and every round still leaves its own
 // statistics.  Results are those of the rounds launched one by one, bit for bit.
+// E = 4 (fp32 only): packs of 4 columns, one Philox block per thread.  A block then holds half
+// the rows at a time, which keeps the rows of all resident blocks within the L2 for up to about
+// 20 devices: the form batches of one-step rounds take (the host decides).  Statistics are then
+// folded over chunks of 1024 columns: equal to the other forms to rounding, not bit for bit.
 // PF = true is a second build that issues the next row's loads before the current row's steps
 // (80 registers, three resident blocks).  With bf16 parameters a row is 48 bytes per thread or
 // less, and when every device runs one or two steps the launch is bound by how many bytes are in

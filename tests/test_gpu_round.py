@@ -289,6 +289,28 @@ def test_batching_rule_on_an_arena_larger_than_the_small_arena_bound(dtype):
     assert batched.h.round_batch() == 2
     single.close()
     batched.close()
+    if dtype == 0:  # fp32, every device one step: the batch takes packs of 4 columns
+        ones = np.ones((5, n), dtype=np.int32)
+        a4, a1 = runtime.Arena(wl), runtime.Arena(wl)
+        a1.h.set_round_batch(1)
+        assert a4.h.last_round_pack() == 0
+        got, launches = _launches(a4, lambda: a4.h.rounds(0, ones, wl.lr, k, a4.select_seed, 2))
+        assert launches == 1 and a4.h.last_round_pack() == 4
+        want = a1.h.rounds(0, ones, wl.lr, k, a1.select_seed, 2)
+        assert a1.h.last_round_pack() == 8 and np.array_equal(got, want)
+        a4.h.synchronize()
+        a1.h.synchronize()
+        assert torch.equal(a4.w, a1.w) and torch.equal(a4.m, a1.m)
+        for back in range(5):
+            x, y = a4.h.stats_read_round(back), (a1.h.stats_read() if back == 0 else None)
+            assert np.all(np.isfinite(x[0])) and np.all(x[1] >= 0)
+            if y is not None:
+                assert np.allclose(x[0], y[0], rtol=2e-6) and np.allclose(x[1], y[1], rtol=2e-6, atol=1e-30)
+        a4.h.rounds(5, steps[:2], wl.lr, k, a4.select_seed, 2)  # two steps somewhere: packs of 8 again
+        assert a4.h.last_round_pack() == 8
+        a4.h.debug_check()
+        a4.close()
+        a1.close()
     if dtype == 1:  # stochastic rounding draws a second random block per pack: launched one by one
         from dataclasses import replace
         sr = runtime.Arena(replace(wl, rounding=1))
