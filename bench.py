@@ -322,16 +322,18 @@ def measure_case(wl, rounds, peak, frac_key, warmup=3):
     # rounds/s with 8 rounds enqueued per library call (hadfl_rounds): small vectors then show the
     # kernel and not the per-call overhead of the caller, while the launch queue stays shallow
     def rounds_by_calls_of_8(r0):
+        arena.run_rounds_fused(r0, 8)  # untimed: the first launch of a kind starts on the previous kernel's cache contents
+        r0 += 8
         launches0 = h.launch_count()
         torch.cuda.synchronize()
         start.record()
-        for i in range(0, 2 * rounds, 8):
-            arena.run_rounds_fused(r0 + i, min(8, 2 * rounds - i))
+        for i in range(0, 4 * rounds, 8):
+            arena.run_rounds_fused(r0 + i, min(8, 4 * rounds - i))
         end.record()
         torch.cuda.synchronize()
-        return start.elapsed_time(end) / (2 * rounds), 2 * rounds / (h.launch_count() - launches0)
+        return start.elapsed_time(end) / (4 * rounds), 4 * rounds / (h.launch_count() - launches0)
     fused_wall_ms, rounds_per_launch = rounds_by_calls_of_8(r)
-    r += 2 * rounds
+    r += 4 * rounds + 8
     # where the library put several rounds into one launch: the same with one launch per round
     single_wall_ms = fused_wall_ms
     if rounds_per_launch > 1:
