@@ -36,8 +36,8 @@
 // other than itself - closed forms, library routines (numpy quantile / mean, scipy normal pdf,
 // torch.optim.SGD, an independent library Philox), brute-force enumeration and the values that
 // follow from Eq. 8 for the paper's two heterogeneity vectors.  Nothing here is "parity
-// unpinned" except what the paper measures on CIFAR-10 (accuracy / time), which this build
-// does not reproduce.
+// unpinned" except what the paper measures on CIFAR-10 (accuracy / time), which is not
+// reproduced here.
 //
 // Precision: parameters and momentum are fp32 with the fused-multiply-add placement spelled
 // out below (compiled with -ffp-contract=off so that only the explicit fmaf calls fuse);
