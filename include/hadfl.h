@@ -216,9 +216,9 @@ int hadfl_rounds(hadfl_handle *h, int64_t first_round, int32_t n_rounds, const i
  * a block takes its columns through all of them before it moves to the next columns, and from the
  * second round on the replicas are read from L2 instead of HBM.  Results - parameters, momentum,
  * counters, selections - are those of the rounds launched one by one, bit for bit; so are every
- * round's statistics, except that large fp32 arenas whose devices all run one step are taken in
- * packs of half the width, which sums the statistics in a different (equally fixed) order: they
- * then agree to rounding.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
+ * round's statistics, except that batches on large fp32 arenas whose devices run at most 1.5 steps
+ * on average are taken in packs of half the width, which sums the statistics in a different
+ * (equally fixed) order: they then agree to rounding.  hadfl_rounds batches the rounds that gain from it (every device runs at most two
  * steps and rounding is to nearest even, or the whole arena - parameters and momentum of all
  * devices - is at most 64 MiB) and launches the others singly.
  * hadfl_set_round_batch: the most rounds per launch, 1 .. 8 (default 8; 1 = never batch);

@@ -267,9 +267,13 @@ int launch_round(hadfl_handle *h, const RoundBatch<NR> &b, float lr) {
     const RoundScratch scratch{h->d_round_partials, h->d_round_group_partials, h->d_round_ticket,
                                h->d_round_stats, h->d_stats};
     int max_steps = 0;
+    int64_t sum_steps = 0, n_rows = 0;
     for (int r = 0; r < b.n_rounds; ++r)
-      for (int j = 0; j < b.round[r].n; ++j)
+      for (int j = 0; j < b.round[r].n; ++j) {
         max_steps = b.round[r].r[j].steps > max_steps ? b.round[r].r[j].steps : max_steps;
+        sum_steps += b.round[r].r[j].steps;
+        ++n_rows;
+      }
     bool launched = false;
     if constexpr (sizeof(WT) == 2) {
       // bf16 parameters and at most two steps per device: the build that prefetches the next row
@@ -279,9 +283,12 @@ int launch_round(hadfl_handle *h, const RoundBatch<NR> &b, float lr) {
             (WT *)h->w, (MT *)h->m, h->cfg.n_params, b, h->keys, step_consts(h, lr), scratch);
       }
     } else if constexpr (NR > 1) {
-      // fp32, a batch in which no device runs more than one step, rows of the resident blocks within
-      // the L2: packs of 4 columns (half the rows in flight per block, twice the blocks).
-      if (max_steps <= 1 && h->round_half_packs) {
+      // fp32, a batch of at most 1.5 steps per device on average (and no device beyond two), rows of
+      // the resident blocks within the L2: packs of 4 columns (half the rows in flight per block,
+      // twice the blocks).  Measured per round, packs of 4 against packs of 8: one step 151 / 181 us
+      // (ResNet-18 size, 8 devices) and 447 / 600 us (2^24, 16 devices); steps 1,2,1,2,... 185 / 190,
+      // 590 / 625 and 520 / 564 us (VGG-16 size); two steps 217 / 209, 690 / 653, 600 / 590 us.
+      if (max_steps <= kRowPerBlockMaxSteps && 2 * sum_steps <= 3 * n_rows && h->round_half_packs) {
         launched = true;
         h->last_launch_pack = E / 2;
         k_round<WT, MT, NormalsFast, E / 2, RM, false, NR><<<h->round_grid_half_packs, kThreads, smem, h->stream>>>(
